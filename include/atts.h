@@ -1,0 +1,161 @@
+/*
+ * libatts - the verification hot path of asynchronous test-time scaling (ATTS) on one B200.
+ *
+ * The target model scores many parallel draft samples, the scores are ranked against an online
+ * calibration set to give conformal p-values, the p-values are thresholded at the rejection rate
+ * alpha, and the calibration set grows by the new scores.
+ *
+ * Conventions for every entry point
+ *   - Pointers marked "dev" are device pointers of the current CUDA device, "host" are host
+ *     pointers.  The caller owns every buffer, workspaces included; the library allocates no
+ *     device memory and keeps no state between calls except a per-process cache of the device's
+ *     properties and one device-side status word.
+ *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     legacy default stream) and returns; results are valid in stream order.  The only call that
+ *     synchronises is atts_last_device_status.
+ *   - The return value is an atts_status.  Argument errors are found before anything is launched
+ *     and leave every output untouched.  There is no CPU or non-sm_100 fallback: on another device
+ *     the calls return ATTS_ERR_ARCH, without a device ATTS_ERR_CUDA.
+ *   - Outputs must not alias inputs.  Sizes of 0 (M, Nc, k) are valid no-ops.
+ *   - Results of the conformal calls are bit-reproducible; atts_score_logprob is bit-reproducible
+ *     for a given shape on a given device (its reduction order is fixed by a static schedule).
+ */
+#ifndef ATTS_H_
+#define ATTS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ATTS_OK = 0,
+  ATTS_ERR_NULL = 1,      /* a required pointer is NULL                                  */
+  ATTS_ERR_SHAPE = 2,     /* a size is negative, too large, or not a supported multiple  */
+  ATTS_ERR_ALIGN = 3,     /* a pointer is not aligned as documented                      */
+  ATTS_ERR_WORKSPACE = 4, /* workspace_bytes is smaller than the matching *_workspace_bytes */
+  ATTS_ERR_CAPACITY = 5,  /* n + k exceeds the calibration buffer's capacity             */
+  ATTS_ERR_ARG = 6,       /* a scalar argument is out of range (alpha, score_mode)       */
+  ATTS_ERR_ARCH = 7,      /* the current device is not sm_100                            */
+  ATTS_ERR_CUDA = 8,      /* a CUDA runtime or driver call failed                        */
+  ATTS_ERR_TIMEOUT = 9    /* reported by atts_last_device_status: a bounded device wait expired */
+} atts_status;
+
+/* Bits of the device status word returned by atts_last_device_status. */
+#define ATTS_DEV_TOKEN_ID_RANGE 1u /* a token id was outside [0, V): that row's log-prob is NaN */
+#define ATTS_DEV_WAIT_EXPIRED 2u   /* a pipeline wait in the scoring kernel ran out; outputs invalid */
+
+/* Stage labels written by atts_classify (the three stages of the rejection-sampling pipeline,
+ * Sec. 3.3): the highest stage a sample reaches in this turn. */
+#define ATTS_STAGE_DRAFT 1    /* nothing was verified (the sample has no score)          */
+#define ATTS_STAGE_ACCEPTED 2 /* verified and p > alpha: the draft continuation is kept  */
+#define ATTS_STAGE_TARGET 3   /* verified and p <= alpha: the target model takes over    */
+
+/* Static string for a status code; never NULL. */
+const char* atts_strerror(int status);
+/* Library version, major * 10000 + minor * 100 + patch. */
+int atts_version(void);
+
+/*
+ * Bytes of workspace atts_score_logprob needs for M rows, hidden size d, vocabulary V and S
+ * samples on the current device.  host out: *bytes.  The figure depends on the device's SM count.
+ */
+int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_t* bytes);
+
+/*
+ * Target-model scoring of draft tokens (Sec. 3.3 "Verification"; the score of Sec. 3.2,
+ * s = -l with l the negative log-likelihood loss of Eq. 2).
+ *
+ * For every row i (one scored draft token): logits z_i = W h_i over the whole vocabulary,
+ * token_logprob[i] = z_i[token_ids[i]] - log sum_v exp(z_i[v]).  The logits are produced tile by
+ * tile on the tensor cores and reduced on the fly; the M x V logit matrix is never written to
+ * memory.  For every sample k (rows seg_offsets[k] .. seg_offsets[k+1]-1):
+ *   score_mode 0: sample_score[k] = -mean(token_logprob)   (mean NLL, the default reading)
+ *              1: -sum     2: +mean     3: +sum;            an empty sample scores NaN.
+ *
+ *   hidden_bf16   dev  [M, d] bf16, row-major, leading dimension d, 16-byte aligned
+ *   lm_head_bf16  dev  [V, d] bf16, row-major (one row per vocabulary entry), 16-byte aligned
+ *   token_ids     dev  [M] int32, each in [0, V); an id outside sets ATTS_DEV_TOKEN_ID_RANGE and
+ *                      yields NaN for that row
+ *   seg_offsets   dev  [S + 1] int32, 0 = o_0 <= o_1 <= ... <= o_S = M (not checked on the device
+ *                      beyond clamping to [0, M])
+ *   M, d, V, S         0 <= M < 2^31, d a multiple of 64 with 64 <= d <= 65536, 1 <= V < 2^31,
+ *                      0 <= S
+ *   token_logprob dev  [M] fp32 out, may be NULL
+ *   sample_score  dev  [S] fp32 out, may be NULL when S == 0
+ *   workspace     dev  256-byte aligned scratch of at least atts_score_workspace_bytes(...);
+ *                      contents are undefined afterwards
+ * Arithmetic: bf16 x bf16 products accumulated in fp32 (tcgen05), fp32 exponentials and sums,
+ * fp64 accumulation of the per-sample sum.
+ */
+int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
+                       const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V, int64_t S,
+                       int32_t score_mode, float* token_logprob, float* sample_score,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Marginal conformal p-value by rank (Eq. p-value, Proposition 1):
+ *   numer[j]  = 1 + #{ i < n : calib_sorted[i] >= scores[j] },  pvalue[j] = numer[j] / (n + 1).
+ * Ties count.  A NaN calibration score (sorted last) counts for every candidate; a NaN candidate
+ * has no score: numer = 0, pvalue = NaN.
+ *
+ *   scores        dev  [Nc] fp32
+ *   calib_sorted  dev  [n] fp32 ascending, NaNs last (as atts_calib_update leaves it); may be NULL
+ *                      when n == 0
+ *   Nc, n              0 <= Nc < 2^31, 0 <= n < 2^24 - 1 (so that n + 1 is exact in fp32)
+ *   numer         dev  [Nc] uint32 out
+ *   pvalue        dev  [Nc] fp32 out (one correctly rounded fp32 division), may be NULL
+ */
+int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
+                        uint32_t* numer, float* pvalue, void* cuda_stream);
+
+/*
+ * Threshold at the rejection rate alpha and ordinal stage label (acceptance rule after
+ * Eq. p-value, Eq. prediction_set, the three stages of Sec. 3.3).  With
+ * k_alpha = floor(alpha * (n + 1)) evaluated in IEEE double on the host:
+ *   numer == 0             -> ATTS_STAGE_DRAFT
+ *   1 <= numer <= k_alpha  -> ATTS_STAGE_TARGET    (p <= alpha)
+ *   otherwise              -> ATTS_STAGE_ACCEPTED  (p >  alpha)
+ *
+ *   numer         dev  [Nc] uint32, as written by atts_conformal_rank for the same n
+ *   alpha              0 < alpha < 1, else ATTS_ERR_ARG
+ *   stage         dev  [Nc] uint8 out
+ *   stage_counts  dev  [3] uint32 out (numbers of samples in stages 1, 2, 3; the third is the
+ *                      budget B of "Budget Prediction"), overwritten; may be NULL
+ */
+int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, uint8_t* stage,
+                  uint32_t* stage_counts, void* cuda_stream);
+
+/* Bytes of workspace atts_calib_update needs to insert k scores into a buffer holding n. */
+int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes);
+
+/*
+ * Online calibration (Sec. 3.2 "Online Calibration"): the calibration set grows by k new scores.
+ * The set is kept as an ascending fp32 array; after the call (in stream order) calib[0 .. n+k) is
+ * the sorted union, as a multiset, of the old n entries and the k new ones.  -0.0 is stored as
+ * +0.0 and every NaN as 0x7FC00000, sorted last, so the result is a unique bit pattern.  Nothing
+ * is evicted.
+ *
+ *   calib         dev  fp32 buffer of `cap` elements, the first n ascending (NaNs last); updated
+ *                      in place
+ *   n, cap, k          0 <= n, 0 <= k, n + k <= cap (else ATTS_ERR_CAPACITY), cap < 2^24 - 1
+ *   new_scores    dev  [k] fp32, any order; may be NULL when k == 0
+ *   n_out         host out, may be NULL: n + k
+ *   workspace     dev  256-byte aligned scratch of at least atts_calib_workspace_bytes(n, k)
+ */
+int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k,
+                      int64_t* n_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Waits for `cuda_stream`, then returns in *bits (host out) the OR of the ATTS_DEV_* conditions
+ * device code has recorded on the current device since the last call, and clears them.  Returns
+ * ATTS_ERR_TIMEOUT if ATTS_DEV_WAIT_EXPIRED is among them, else ATTS_OK.
+ */
+int atts_last_device_status(void* cuda_stream, uint32_t* bits);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTS_H_ */

@@ -1,0 +1,144 @@
+"""Thin Python binding of libatts (ctypes): argument marshalling only.
+
+Every function takes torch CUDA tensors, passes their device pointers and the current
+CUDA stream to the C entry point of the same name (include/atts.h), and raises
+:class:`AttsError` on a non-zero status.  Nothing is computed here, and there is no
+fallback: if the CUDA library cannot be loaded, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_double, c_int, c_int32, c_int64, c_size_t, c_void_p, c_char_p, POINTER, c_uint32
+
+from . import build as _build
+
+EXPORTS = (
+    "atts_strerror", "atts_version", "atts_score_workspace_bytes", "atts_score_logprob",
+    "atts_conformal_rank", "atts_classify", "atts_calib_workspace_bytes", "atts_calib_update",
+    "atts_last_device_status",
+)
+
+STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
+DEV_TOKEN_ID_RANGE, DEV_WAIT_EXPIRED = 1, 2
+
+_lib = None
+
+
+class AttsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {strerror(status)} (status {status})")
+
+
+def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
+    """Load libatts.so from the package directory (building it first if the sources are newer)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if rebuild_if_stale and _build.is_stale():
+        try:
+            _build.build_library()
+        except Exception:
+            if not os.path.exists(path):
+                raise
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_2509_15148_b200.build`")
+    lib = ctypes.CDLL(path)
+    lib.atts_strerror.restype = c_char_p
+    lib.atts_strerror.argtypes = [c_int]
+    lib.atts_version.restype = c_int
+    lib.atts_score_workspace_bytes.argtypes = [c_int64, c_int64, c_int64, c_int64, POINTER(c_size_t)]
+    lib.atts_score_logprob.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64,
+                                       c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.atts_conformal_rank.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_void_p]
+    lib.atts_classify.argtypes = [c_void_p, c_int64, c_int64, c_double, c_void_p, c_void_p, c_void_p]
+    lib.atts_calib_workspace_bytes.argtypes = [c_int64, c_int64, POINTER(c_size_t)]
+    lib.atts_calib_update.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
+                                      c_size_t, c_void_p]
+    lib.atts_last_device_status.argtypes = [c_void_p, POINTER(c_uint32)]
+    for name in EXPORTS[2:]:
+        getattr(lib, name).restype = c_int
+    _lib = lib
+    return lib
+
+
+def strerror(status: int) -> str:
+    return load().atts_strerror(int(status)).decode()
+
+
+def version() -> int:
+    return load().atts_version()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise AttsError(status, where)
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def score_workspace_bytes(M: int, d: int, V: int, S: int) -> int:
+    out = c_size_t(0)
+    _check(load().atts_score_workspace_bytes(M, d, V, S, ctypes.byref(out)), "atts_score_workspace_bytes")
+    return out.value
+
+
+def score_logprob(hidden, lm_head, token_ids, seg_offsets, token_logprob, sample_score, workspace,
+                  score_mode: int = 0) -> None:
+    """hidden [M,d] bf16, lm_head [V,d] bf16, token_ids [M] i32, seg_offsets [S+1] i32 ->
+    token_logprob [M] f32 (or None), sample_score [S] f32; workspace: uint8 tensor."""
+    M, d = hidden.shape
+    V = lm_head.shape[0]
+    S = seg_offsets.numel() - 1
+    _check(load().atts_score_logprob(_ptr(hidden), _ptr(lm_head), _ptr(token_ids), _ptr(seg_offsets), M, d, V, S,
+                                     score_mode, _ptr(token_logprob), _ptr(sample_score), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream()), "atts_score_logprob")
+
+
+def conformal_rank(scores, calib_sorted, n: int, numer, pvalue=None) -> None:
+    """scores [Nc] f32, calib_sorted (first n entries used) -> numer [Nc] u32 (int32 storage), pvalue [Nc] f32."""
+    _check(load().atts_conformal_rank(_ptr(scores), scores.numel(), _ptr(calib_sorted), n, _ptr(numer), _ptr(pvalue),
+                                      _stream()), "atts_conformal_rank")
+
+
+def classify(numer, n: int, alpha: float, stage, stage_counts=None) -> None:
+    """numer [Nc] u32 -> stage [Nc] u8, stage_counts [3] u32 (int32 storage) or None."""
+    _check(load().atts_classify(_ptr(numer), numer.numel(), n, float(alpha), _ptr(stage), _ptr(stage_counts),
+                                _stream()), "atts_classify")
+
+
+def calib_workspace_bytes(n: int, k: int) -> int:
+    out = c_size_t(0)
+    _check(load().atts_calib_workspace_bytes(n, k, ctypes.byref(out)), "atts_calib_workspace_bytes")
+    return out.value
+
+
+def calib_update(calib, n: int, new_scores, workspace) -> int:
+    """calib: f32 buffer of capacity calib.numel() whose first n entries are sorted; inserts new_scores in place.
+    Returns the new fill n + k."""
+    n_out = c_int64(0)
+    k = 0 if new_scores is None else new_scores.numel()
+    _check(load().atts_calib_update(_ptr(calib), n, calib.numel(), _ptr(new_scores), k, ctypes.byref(n_out),
+                                    _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _stream()), "atts_calib_update")
+    return n_out.value
+
+
+def last_device_status() -> int:
+    """Synchronises the current stream; returns and clears the device status bits. Raises on an expired wait."""
+    bits = c_uint32(0)
+    st = load().atts_last_device_status(_stream(), ctypes.byref(bits))
+    if st not in (0, 9):
+        raise AttsError(st, "atts_last_device_status")
+    if st == 9:
+        raise AttsError(st, "atts_last_device_status")
+    return bits.value

@@ -1,0 +1,302 @@
+// C-ABI entry points of libatts (declared in include/atts.h): argument checks, launch geometry,
+// tensor-map encoding.  All device work is in the kernels of conformal.cuh and lmhead_lse.cuh.
+#include "atts.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+#include <math.h>
+#include <mutex>
+
+#include "conformal.cuh"
+#include "lmhead_lse.cuh"
+
+namespace atts {
+
+__device__ unsigned int g_dev_status = 0u;
+
+struct DeviceInfo {
+  bool ready = false;
+  int status = ATTS_OK;  // sticky result of the probe
+  int sm_count = 0;
+  unsigned int* dev_status = nullptr;
+  PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+};
+
+static DeviceInfo g_info[64];
+static std::mutex g_mu;
+
+// Probes the current device once: architecture, SM count, address of the status word, driver entry
+// point for tensor-map encoding, and the opt-in shared-memory sizes of the kernels.
+static int device_info(const DeviceInfo** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceInfo& di = g_info[dev];
+  if (!di.ready) {
+    di.ready = true;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+      di.status = ATTS_ERR_CUDA;
+    } else if (major != 10) {
+      di.status = ATTS_ERR_ARCH;
+    } else {
+      bool ok = cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
+      ok = ok && cudaGetSymbolAddress((void**)&di.dev_status, g_dev_status) == cudaSuccess;
+      cudaDriverEntryPointQueryResult q;
+      void* fn = nullptr;
+      ok = ok && cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+           q == cudaDriverEntryPointSuccess && fn != nullptr;
+      di.encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+      ok = ok && cudaFuncSetAttribute(lmhead_lse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kScoreSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kSortMaxK * 4) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kSortMaxK * 4) == cudaSuccess;
+      if (!ok) {
+        cudaGetLastError();
+        di.status = ATTS_ERR_CUDA;
+      }
+    }
+  }
+  *out = &di;
+  return di.status;
+}
+
+static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int launch_status() { return cudaGetLastError() == cudaSuccess ? ATTS_OK : ATTS_ERR_CUDA; }
+
+// Workspace layout of atts_score_logprob: [partials C * M_pad float2][gathered M_pad f32][logprob M_pad f32]
+struct ScoreWs {
+  size_t partial_off, gathered_off, logprob_off, total;
+};
+static ScoreWs score_ws(const ScorePlan& p) {
+  ScoreWs w;
+  w.partial_off = 0;
+  w.gathered_off = round_up((size_t)p.C * p.M_pad * sizeof(float2), 256);
+  w.logprob_off = w.gathered_off + round_up((size_t)p.M_pad * sizeof(float), 256);
+  w.total = w.logprob_off + round_up((size_t)p.M_pad * sizeof(float), 256);
+  if (w.total == 0) w.total = 256;
+  return w;
+}
+
+static int check_score_shape(int64_t M, int64_t d, int64_t V, int64_t S) {
+  if (M < 0 || M >= (1ll << 31) - kBlockM || S < 0 || S >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  if (d < 64 || d > 65536 || d % 64 != 0) return ATTS_ERR_SHAPE;
+  if (V < 1 || V >= (1ll << 31) - kBlockN) return ATTS_ERR_SHAPE;
+  return ATTS_OK;
+}
+
+static int encode_2d(const DeviceInfo* di, CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = di->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ATTS_OK : ATTS_ERR_CUDA;
+}
+
+}  // namespace atts
+
+using namespace atts;
+
+extern "C" {
+
+const char* atts_strerror(int status) {
+  switch (status) {
+    case ATTS_OK: return "ok";
+    case ATTS_ERR_NULL: return "a required pointer is NULL";
+    case ATTS_ERR_SHAPE: return "a size is negative, too large or not a supported multiple";
+    case ATTS_ERR_ALIGN: return "a pointer is not aligned as required";
+    case ATTS_ERR_WORKSPACE: return "the workspace is too small";
+    case ATTS_ERR_CAPACITY: return "n + k exceeds the calibration buffer's capacity";
+    case ATTS_ERR_ARG: return "a scalar argument is out of range";
+    case ATTS_ERR_ARCH: return "the current device is not sm_100 (no fallback path exists)";
+    case ATTS_ERR_CUDA: return "a CUDA call failed (no usable device?)";
+    case ATTS_ERR_TIMEOUT: return "a bounded wait on the device expired";
+    default: return "unknown status";
+  }
+}
+
+int atts_version(void) { return 100; }
+
+int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_t* bytes) {
+  if (!bytes) return ATTS_ERR_NULL;
+  int st = check_score_shape(M, d, V, S);
+  if (st != ATTS_OK) return st;
+  const DeviceInfo* di;
+  st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  *bytes = score_ws(make_score_plan(M, d, V, di->sm_count)).total;
+  return ATTS_OK;
+}
+
+int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
+                       const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V, int64_t S, int32_t score_mode,
+                       float* token_logprob, float* sample_score, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream) {
+  int st = check_score_shape(M, d, V, S);
+  if (st != ATTS_OK) return st;
+  if (score_mode < 0 || score_mode > 3) return ATTS_ERR_ARG;
+  if (!lm_head_bf16 || !seg_offsets || !workspace) return ATTS_ERR_NULL;
+  if (M > 0 && (!hidden_bf16 || !token_ids)) return ATTS_ERR_NULL;
+  if (S > 0 && !sample_score) return ATTS_ERR_NULL;
+  if (!aligned(hidden_bf16, 16) || !aligned(lm_head_bf16, 16) || !aligned(workspace, 256) ||
+      !aligned(token_ids, 4) || !aligned(seg_offsets, 4) || !aligned(token_logprob, 4) || !aligned(sample_score, 4))
+    return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  const ScorePlan plan = make_score_plan(M, d, V, di->sm_count);
+  const ScoreWs ws = score_ws(plan);
+  if (workspace_bytes < ws.total) return ATTS_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* wsp = static_cast<uint8_t*>(workspace);
+  float2* partial = reinterpret_cast<float2*>(wsp + ws.partial_off);
+  float* gathered = reinterpret_cast<float*>(wsp + ws.gathered_off);
+  float* logprob_ws = reinterpret_cast<float*>(wsp + ws.logprob_off);
+
+  if (M > 0) {
+    CUtensorMap map_h, map_w;
+    if (encode_2d(di, &map_h, hidden_bf16, M, d, kBlockM) != ATTS_OK) return ATTS_ERR_CUDA;
+    if (encode_2d(di, &map_w, lm_head_bf16, V, d, kBlockN) != ATTS_OK) return ATTS_ERR_CUDA;
+    const int grid = plan.units < di->sm_count ? plan.units : di->sm_count;
+    lmhead_lse_kernel<<<grid, kScoreThreads, kScoreSmemBytes, stream>>>(map_h, map_w, token_ids, plan, partial,
+                                                                        gathered, di->dev_status);
+    if ((st = launch_status()) != ATTS_OK) return st;
+    lse_combine_kernel<<<(unsigned)((M + 255) / 256), 256, 0, stream>>>(partial, gathered, token_ids, (int)M, plan.M_pad,
+                                                                        plan.C, (int)V, logprob_ws, token_logprob,
+                                                                        di->dev_status);
+    if ((st = launch_status()) != ATTS_OK) return st;
+  }
+  if (S > 0) {
+    segment_score_kernel<<<(unsigned)S, 256, 0, stream>>>(logprob_ws, seg_offsets, (int)M, (int)S, score_mode, sample_score);
+    if ((st = launch_status()) != ATTS_OK) return st;
+  }
+  return ATTS_OK;
+}
+
+int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n, uint32_t* numer,
+                        float* pvalue, void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  if (Nc > 0 && (!scores || !numer)) return ATTS_ERR_NULL;
+  if (n > 0 && !calib_sorted) return ATTS_ERR_NULL;
+  if (!aligned(scores, 16) || !aligned(numer, 16) || !aligned(pvalue, 16) || !aligned(calib_sorted, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  if (Nc == 0) return ATTS_OK;
+  // Splitter level: whole buffer in shared memory up to 8192 entries, else every 2^L-th entry with
+  // at most 2048 splitters.
+  int L = 0;
+  if (n > 8192)
+    while (((n + (1ll << L) - 1) >> L) > 2048) ++L;
+  const int ns = (int)((n + (1ll << L) - 1) >> L);
+  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
+  int64_t blocks = (Nc + per_block - 1) / per_block;
+  const int64_t max_blocks = (int64_t)di->sm_count * 8;
+  if (blocks > max_blocks) blocks = max_blocks;
+  rank_kernel<<<(unsigned)blocks, kRankThreads, (size_t)ns * 4, static_cast<cudaStream_t>(cuda_stream)>>>(
+      scores, Nc, calib_sorted, (int)n, ns, L, numer, pvalue);
+  return launch_status();
+}
+
+int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, uint8_t* stage, uint32_t* stage_counts,
+                  void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  if (!(alpha > 0.0 && alpha < 1.0)) return ATTS_ERR_ARG;
+  if (Nc > 0 && (!numer || !stage)) return ATTS_ERR_NULL;
+  if (!aligned(numer, 16) || !aligned(stage, 16) || !aligned(stage_counts, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (stage_counts && cudaMemsetAsync(stage_counts, 0, 3 * sizeof(uint32_t), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  if (Nc == 0) return ATTS_OK;
+  const uint32_t k_alpha = (uint32_t)floor(alpha * (double)(n + 1));
+  const int64_t per_block = (int64_t)kClassifyThreads * kClassifyPerThread;
+  int64_t blocks = (Nc + per_block - 1) / per_block;
+  const int64_t max_blocks = (int64_t)di->sm_count * 8;
+  if (blocks > max_blocks) blocks = max_blocks;
+  classify_kernel<<<(unsigned)blocks, kClassifyThreads, 0, stream>>>(numer, Nc, k_alpha, stage, stage_counts);
+  return launch_status();
+}
+
+// Workspace of atts_calib_update: [sorted new keys: min(k, kSortMaxK) u32][merged copy: n + k f32]
+int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes) {
+  if (!bytes) return ATTS_ERR_NULL;
+  if (n < 0 || k < 0 || n + k >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
+  *bytes = round_up((size_t)kk * 4, 256) + round_up((size_t)(n + k) * 4, 256) + 256;
+  return ATTS_OK;
+}
+
+int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (n < 0 || k < 0 || cap < 0 || cap >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  if (n + k > cap) return ATTS_ERR_CAPACITY;
+  if ((cap > 0 && !calib) || (k > 0 && (!new_scores || !workspace))) return ATTS_ERR_NULL;
+  if (!aligned(calib, 4) || !aligned(new_scores, 4) || !aligned(workspace, 256)) return ATTS_ERR_ALIGN;
+  size_t need = 0;
+  atts_calib_workspace_bytes(n, k, &need);
+  if (k > 0 && workspace_bytes < need) return ATTS_ERR_WORKSPACE;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  if (n_out) *n_out = n + k;
+  if (k == 0) return ATTS_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
+  uint32_t* sorted_keys = static_cast<uint32_t*>(workspace);
+  float* merged = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up((size_t)kk * 4, 256));
+  // Batches larger than one sort launch handles are inserted slice by slice.
+  int64_t cur = n;
+  for (int64_t off = 0; off < k; off += kSortMaxK) {
+    const int kc = (int)((k - off) < kSortMaxK ? (k - off) : kSortMaxK);
+    int sort_blocks = (kc + 7) / 8;
+    if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
+    sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)kc * 4, stream>>>(new_scores + off, kc, sorted_keys);
+    if ((st = launch_status()) != ATTS_OK) return st;
+    int64_t total = cur + kc;
+    int merge_blocks = (int)((total + kMergeThreads - 1) / kMergeThreads);
+    if (merge_blocks > di->sm_count * 4) merge_blocks = di->sm_count * 4;
+    merge_kernel<<<merge_blocks, kMergeThreads, (size_t)kc * 4, stream>>>(calib, (int)cur, sorted_keys, kc, merged);
+    if ((st = launch_status()) != ATTS_OK) return st;
+    if (cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+      cudaGetLastError();
+      return ATTS_ERR_CUDA;
+    }
+    cur = total;
+  }
+  return ATTS_OK;
+}
+
+int atts_last_device_status(void* cuda_stream, uint32_t* bits) {
+  if (!bits) return ATTS_ERR_NULL;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  unsigned int v = 0;
+  if (cudaMemcpyAsync(&v, di->dev_status, sizeof(v), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemsetAsync(di->dev_status, 0, sizeof(v), stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  *bits = v;
+  return (v & ATTS_DEV_WAIT_EXPIRED) ? ATTS_ERR_TIMEOUT : ATTS_OK;
+}
+
+}  // extern "C"

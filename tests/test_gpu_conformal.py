@@ -1,0 +1,180 @@
+"""GPU parity: rank / p-value, classify and calibration update through the C-ABI, against the CPU
+oracle, bit for bit, on the same fp32 score arrays."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import atts_oracle as orc
+from paper_2509_15148_b200 import binding, inputs
+from tests.gpu_util import dev, f32_bits, host_u32, poison, workspace
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_rank(scores: np.ndarray, calib: np.ndarray, want_p=True):
+    s, c = dev(scores), dev(calib) if calib.size else None
+    numer = poison((scores.size,), torch.int32)
+    p = poison((scores.size,), torch.float32) if want_p else None
+    binding.conformal_rank(s, c, calib.size, numer, p)
+    torch.cuda.synchronize()
+    return host_u32(numer), (p.cpu().numpy() if want_p else None)
+
+
+def gpu_classify(numer: np.ndarray, n: int, alpha: float):
+    nm = dev(numer)
+    stage = poison((numer.size,), torch.uint8)
+    counts = poison((3,), torch.int32)
+    binding.classify(nm, n, alpha, stage, counts)
+    torch.cuda.synchronize()
+    return stage.cpu().numpy(), host_u32(counts)
+
+
+def gpu_update(calib: np.ndarray, new: np.ndarray, cap: int):
+    buf = poison((cap,), torch.float32)
+    buf[:calib.size] = dev(calib) if calib.size else buf[:0]
+    ws = workspace(binding.calib_workspace_bytes(calib.size, new.size))
+    n2 = binding.calib_update(buf, calib.size, dev(new) if new.size else None, ws)
+    torch.cuda.synchronize()
+    return buf.cpu().numpy(), n2
+
+
+def check_rank(scores, calib):
+    numer, p = gpu_rank(scores, calib)
+    want = orc.conformal_numer_sorted(scores, calib)
+    assert np.array_equal(numer, want)
+    assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want, calib.size)))
+    return numer
+
+
+@pytest.mark.parametrize("Nc,n", [(1, 1), (5, 0), (1023, 7), (4096, 256), (4099, 8192), (70001, 8193),
+                                   (33333, 65536), (20011, 327680), (1000, 1000001)])
+def test_rank_pvalue_bit_exact(Nc, n):
+    scores = inputs.lognormal_scores(100 + Nc, Nc)
+    calib = np.sort(inputs.lognormal_scores(200 + n, n))
+    numer = check_rank(scores, calib)
+    # sampled outputs against the literal double-sum definition
+    idx = np.random.default_rng(0).choice(Nc, size=min(Nc, 64), replace=False)
+    assert np.array_equal(numer[idx], orc.conformal_numer_count(scores[idx], calib))
+
+
+def test_rank_ties_extremes_and_special_values():
+    calib = np.sort(np.round(inputs.lognormal_scores(1, 50000), 1))     # heavy ties
+    scores = np.concatenate([np.round(inputs.lognormal_scores(2, 9000), 1), calib[::97],
+                             np.array([0.0, -0.0, -1.0, 1e30, np.inf, -np.inf, np.nan], np.float32)])
+    check_rank(scores, calib)
+    calib = orc.calib_update(np.zeros(0, np.float32),
+                             np.array([-np.inf, -1.0, -0.0, 0.0, 5.0, np.inf, np.nan, np.nan], np.float32))
+    scores = np.array([np.nan, 0.0, -0.0, np.inf, -np.inf, 6.0, 5.0, -1.0], np.float32)
+    numer = check_rank(scores, calib)
+    assert np.array_equal(numer, orc.conformal_numer_count(scores, calib))
+    # every score of the buffer ranked against itself: n - i + 1 for distinct values
+    calib = np.unique(inputs.lognormal_scores(3, 20000))
+    numer, _ = gpu_rank(calib, calib)
+    assert np.array_equal(numer, np.arange(calib.size + 1, 1, -1, dtype=np.uint32))
+
+
+def test_rank_without_pvalue_output_and_empty_input():
+    calib = np.sort(inputs.lognormal_scores(5, 300))
+    scores = inputs.lognormal_scores(6, 77)
+    numer, _ = gpu_rank(scores, calib, want_p=False)
+    assert np.array_equal(numer, orc.conformal_numer_sorted(scores, calib))
+    binding.conformal_rank(torch.empty(0, device="cuda"), dev(calib), calib.size, torch.empty(0, dtype=torch.int32, device="cuda"))
+
+
+@pytest.mark.parametrize("alpha", [0.05, 0.1, 0.2, 0.25, 0.4, 0.999])
+@pytest.mark.parametrize("Nc,n", [(3, 9), (4096 + 5, 255), (100000, 65536)])
+def test_classify_bit_exact(alpha, Nc, n):
+    rng = np.random.default_rng(Nc + n)
+    numer = rng.integers(0, n + 2, size=Nc).astype(np.uint32)
+    ka = orc.k_alpha(alpha, n)
+    numer[: min(Nc, 3)] = np.array([ka, ka + 1, 0], np.uint32)[: min(Nc, 3)]     # both sides of the threshold
+    stage, counts = gpu_classify(numer, n, alpha)
+    want_stage, want_counts = orc.classify(numer, n, alpha)
+    assert np.array_equal(stage, want_stage)
+    assert np.array_equal(counts, want_counts)
+
+
+def test_classify_boundary_cases_and_no_counts():
+    stage, counts = gpu_classify(np.array([1, 2], np.uint32), 9, 0.1)     # alpha (n + 1) = 1 exactly
+    assert stage.tolist() == [3, 2] and counts.tolist() == [0, 1, 1]
+    stage, counts = gpu_classify(np.array([1, 2, 9], np.uint32), 8, 0.1)  # k_alpha = 0: nobody rejected
+    assert stage.tolist() == [2, 2, 2] and counts.tolist() == [0, 3, 0]
+    numer = dev(np.arange(40, dtype=np.uint32))
+    stage = poison((40,), torch.uint8)
+    binding.classify(numer, 50, 0.25, stage, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(stage.cpu().numpy(), orc.classify(np.arange(40, dtype=np.uint32), 50, 0.25)[0])
+    counts = poison((3,), torch.int32)
+    binding.classify(numer[:0], 50, 0.25, stage[:0], counts)              # empty input still zeroes the counts
+    torch.cuda.synchronize()
+    assert host_u32(counts).tolist() == [0, 0, 0]
+
+
+@pytest.mark.parametrize("n,k", [(0, 1), (0, 300), (1, 1), (256, 8), (4096, 64), (1000, 4097), (65536, 4096),
+                                  (323584, 4096), (5000, 16384), (100, 40000), (7, 0)])
+def test_calib_update_bit_exact(n, k):
+    calib = np.sort(inputs.lognormal_scores(300 + n, n))
+    new = inputs.lognormal_scores(400 + k, k)
+    buf, n2 = gpu_update(calib, new, n + k + 5)
+    assert n2 == n + k
+    want = orc.calib_update(calib, new)
+    assert np.array_equal(f32_bits(buf[:n2]), f32_bits(want))
+    assert np.all(f32_bits(buf[n2:]) == 0xFFFFFFFF)     # nothing written past the new fill
+
+
+def test_calib_update_duplicates_and_special_values():
+    calib = orc.calib_update(np.zeros(0, np.float32), np.round(inputs.lognormal_scores(1, 3000), 1))
+    weird_nan = np.array([0x7F800001, 0xFFC00123], np.uint32).view(np.float32)
+    new = np.concatenate([np.round(inputs.lognormal_scores(2, 500), 1),
+                          np.array([-0.0, 0.0, np.inf, -np.inf, 3.0, 3.0], np.float32), weird_nan])
+    buf, n2 = gpu_update(calib, new, calib.size + new.size)
+    assert np.array_equal(f32_bits(buf[:n2]), f32_bits(orc.calib_update(calib, new)))
+    # a second insert on top of a buffer that already holds NaNs
+    buf2, n3 = gpu_update(buf[:n2], new, n2 + new.size)
+    assert np.array_equal(f32_bits(buf2[:n3]), f32_bits(orc.calib_update(buf[:n2], new)))
+
+
+def test_calib_update_capacity_error_leaves_buffer_untouched():
+    buf = dev(np.sort(inputs.lognormal_scores(1, 16)))
+    before = buf.clone()
+    ws = workspace(binding.calib_workspace_bytes(16, 4))
+    with pytest.raises(binding.AttsError) as e:
+        binding.calib_update(buf, 16, dev(inputs.lognormal_scores(2, 4)), ws)
+    assert e.value.status == 5
+    torch.cuda.synchronize()
+    assert torch.equal(buf, before)
+
+
+def test_conformal_stress_sequence_bit_exact():
+    """The conformal-only workload at reduced length: rank, classify at three alphas, merge-insert, repeated,
+    every step's outputs against the oracle."""
+    cfg = inputs.CONFORMAL_STRESS
+    Nc, n0, k, steps = cfg["Nc"], cfg["n0"], cfg["k"], 6
+    scores = inputs.lognormal_scores(inputs.BASE_SEED + 1, Nc)
+    calib = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, n0))
+    cap = n0 + k * steps
+    buf = poison((cap,), torch.float32)
+    buf[:n0] = dev(calib)
+    s_dev = dev(scores)
+    numer = poison((Nc,), torch.int32)
+    p = poison((Nc,), torch.float32)
+    stage = poison((Nc,), torch.uint8)
+    counts = poison((3,), torch.int32)
+    ws = workspace(binding.calib_workspace_bytes(cap, k))
+    n = n0
+    for t in range(steps):
+        binding.conformal_rank(s_dev, buf, n, numer, p)
+        want_numer = orc.conformal_numer_sorted(scores, calib)
+        assert np.array_equal(host_u32(numer), want_numer)
+        assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, n)))
+        for alpha in cfg["alphas"]:
+            binding.classify(numer, n, alpha, stage, counts)
+            want_stage, want_counts = orc.classify(want_numer, n, alpha)
+            assert np.array_equal(stage.cpu().numpy(), want_stage)
+            assert np.array_equal(host_u32(counts), want_counts)
+        new = inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, k)
+        n = binding.calib_update(buf, n, dev(new), ws)
+        calib = orc.calib_update(calib, new)
+        assert n == calib.size
+        assert np.array_equal(f32_bits(buf[:n]), f32_bits(calib))
+    assert binding.last_device_status() == 0
