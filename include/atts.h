@@ -155,6 +155,17 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
  */
 int atts_last_device_status(void* cuda_stream, uint32_t* bits);
 
+/*
+ * Timing hooks (measurement aid; the paper has no counterpart).  Between atts_profile_begin and
+ * atts_profile_end every atts_score_logprob call records a pair of CUDA events on its stream
+ * directly around the fused LM-head kernel, for at most `max_records` calls (<= 4096).
+ * atts_profile_end waits for the recorded events, writes the kernel durations in milliseconds to
+ * ms[0 .. min(*count, cap)) (host), sets *count (host) to the number of recorded launches and
+ * releases the events.  Not thread-safe; one profiling session per process at a time.
+ */
+int atts_profile_begin(int max_records);
+int atts_profile_end(float* ms, int cap, int* count);
+
 #ifdef __cplusplus
 }
 #endif

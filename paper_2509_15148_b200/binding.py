@@ -16,7 +16,7 @@ from . import build as _build
 EXPORTS = (
     "atts_strerror", "atts_version", "atts_score_workspace_bytes", "atts_score_logprob",
     "atts_conformal_rank", "atts_classify", "atts_calib_workspace_bytes", "atts_calib_update",
-    "atts_last_device_status",
+    "atts_last_device_status", "atts_profile_begin", "atts_profile_end",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -58,6 +58,8 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.atts_calib_update.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
                                       c_size_t, c_void_p]
     lib.atts_last_device_status.argtypes = [c_void_p, POINTER(c_uint32)]
+    lib.atts_profile_begin.argtypes = [c_int]
+    lib.atts_profile_end.argtypes = [POINTER(ctypes.c_float), c_int, POINTER(c_int)]
     for name in EXPORTS[2:]:
         getattr(lib, name).restype = c_int
     _lib = lib
@@ -142,3 +144,16 @@ def last_device_status() -> int:
     if st == 9:
         raise AttsError(st, "atts_last_device_status")
     return bits.value
+
+
+def profile_begin(max_records: int = 1024) -> None:
+    """Start recording CUDA-event pairs around the fused scoring kernel of every score_logprob call."""
+    _check(load().atts_profile_begin(int(max_records)), "atts_profile_begin")
+
+
+def profile_end(cap: int = 4096) -> list[float]:
+    """Stop recording; returns the fused kernel's durations in milliseconds, one per recorded call."""
+    buf = (ctypes.c_float * cap)()
+    cnt = c_int(0)
+    _check(load().atts_profile_end(buf, cap, ctypes.byref(cnt)), "atts_profile_end")
+    return [float(buf[i]) for i in range(min(cnt.value, cap))]

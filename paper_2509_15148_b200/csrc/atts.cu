@@ -68,6 +68,14 @@ static int device_info(const DeviceInfo** out) {
   return di.status;
 }
 
+// Timing hooks: event pairs recorded around the fused kernel while a profiling session is open.
+struct Profile {
+  bool on = false;
+  int cap = 0, used = 0;
+  cudaEvent_t* ev = nullptr;  // 2 * cap events
+};
+static Profile g_prof;
+
 static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int launch_status() { return cudaGetLastError() == cudaSuccess ? ATTS_OK : ATTS_ERR_CUDA; }
@@ -169,8 +177,11 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
     if (encode_2d(di, &map_h, hidden_bf16, M, d, kBlockM) != ATTS_OK) return ATTS_ERR_CUDA;
     if (encode_2d(di, &map_w, lm_head_bf16, V, d, kBlockN) != ATTS_OK) return ATTS_ERR_CUDA;
     const int grid = plan.units < di->sm_count ? plan.units : di->sm_count;
+    const bool timed = g_prof.on && g_prof.used < g_prof.cap;
+    if (timed) cudaEventRecord(g_prof.ev[2 * g_prof.used], stream);
     lmhead_lse_kernel<<<grid, kScoreThreads, kScoreSmemBytes, stream>>>(map_h, map_w, token_ids, plan, partial,
                                                                         gathered, di->dev_status);
+    if (timed) cudaEventRecord(g_prof.ev[2 * g_prof.used++ + 1], stream);
     if ((st = launch_status()) != ATTS_OK) return st;
     lse_combine_kernel<<<(unsigned)((M + 255) / 256), 256, 0, stream>>>(partial, gathered, token_ids, (int)M, plan.M_pad,
                                                                         plan.C, (int)V, logprob_ws, token_logprob,
@@ -297,6 +308,48 @@ int atts_last_device_status(void* cuda_stream, uint32_t* bits) {
   }
   *bits = v;
   return (v & ATTS_DEV_WAIT_EXPIRED) ? ATTS_ERR_TIMEOUT : ATTS_OK;
+}
+
+int atts_profile_begin(int max_records) {
+  if (max_records < 1 || max_records > 4096) return ATTS_ERR_ARG;
+  if (g_prof.on) return ATTS_ERR_ARG;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  g_prof.ev = new cudaEvent_t[2 * max_records];
+  for (int i = 0; i < 2 * max_records; ++i) {
+    if (cudaEventCreate(&g_prof.ev[i]) != cudaSuccess) {
+      for (int j = 0; j < i; ++j) cudaEventDestroy(g_prof.ev[j]);
+      delete[] g_prof.ev;
+      g_prof.ev = nullptr;
+      cudaGetLastError();
+      return ATTS_ERR_CUDA;
+    }
+  }
+  g_prof.cap = max_records;
+  g_prof.used = 0;
+  g_prof.on = true;
+  return ATTS_OK;
+}
+
+int atts_profile_end(float* ms, int cap, int* count) {
+  if (!count || (cap > 0 && !ms)) return ATTS_ERR_NULL;
+  if (!g_prof.on) return ATTS_ERR_ARG;
+  int st = ATTS_OK;
+  for (int i = 0; i < g_prof.used; ++i) {
+    float t = 0.f;
+    if (cudaEventSynchronize(g_prof.ev[2 * i + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&t, g_prof.ev[2 * i], g_prof.ev[2 * i + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      st = ATTS_ERR_CUDA;
+    }
+    if (i < cap) ms[i] = t;
+  }
+  *count = g_prof.used;
+  for (int i = 0; i < 2 * g_prof.cap; ++i) cudaEventDestroy(g_prof.ev[i]);
+  delete[] g_prof.ev;
+  g_prof = Profile{};
+  return st;
 }
 
 }  // extern "C"
