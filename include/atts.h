@@ -40,7 +40,8 @@ typedef enum {
   ATTS_ERR_ARG = 6,       /* a scalar argument is out of range (alpha, score_mode)       */
   ATTS_ERR_ARCH = 7,      /* the current device is not sm_100                            */
   ATTS_ERR_CUDA = 8,      /* a CUDA runtime or driver call failed                        */
-  ATTS_ERR_TIMEOUT = 9    /* reported by atts_last_device_status: a bounded device wait expired */
+  ATTS_ERR_TIMEOUT = 9,   /* reported by atts_last_device_status: a bounded device wait expired */
+  ATTS_ERR_SCRATCH_LIMIT = 10 /* atts_calib_update_static: the sizes exceed its built-in scratch */
 } atts_status;
 
 /* Bits of the device status word returned by atts_last_device_status. */
@@ -147,6 +148,39 @@ int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes);
  */
 int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k,
                       int64_t* n_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Allocation-free variant of atts_calib_update (a convenience of this library; the paper has no
+ * counterpart).  Same result, bit for bit, but the caller passes no workspace: the scratch is a
+ * fixed array inside the library's device image.
+ *
+ * Who this is for: code that runs where device memory can no longer be obtained - a plug-in of a
+ * serving engine that has claimed nearly all of HBM for its KV cache at start-up, a control loop
+ * that must not call cudaMalloc because that call synchronises the whole device and would stall the
+ * asynchronous pipeline this method exists to keep busy, or a component that is simply handed a
+ * stream and a few pointers and owns no allocator.  This entry point never calls cudaMalloc,
+ * cudaFree or any other allocating routine.
+ *
+ * Limits: n + k <= ATTS_STATIC_MAX_TOTAL and k <= ATTS_STATIC_MAX_NEW, else
+ * ATTS_ERR_SCRATCH_LIMIT and nothing is launched (use atts_calib_update with a workspace then).
+ * Cost: every device that loads the library holds the array (ATTS_STATIC_SCRATCH_BYTES) until the
+ * process exits, whether or not this entry point is ever called.
+ *
+ * Set-up: the first call on each device looks up the array's device address (with that device
+ * current).  Make that first call during start-up, before any stream capture is begun.
+ * Sharing: all calls on a device use the same array, and it keeps whatever the last call left in
+ * it.  Nothing in it needs to start at zero (each call overwrites every element it later reads),
+ * but two calls whose work overlaps on the GPU - different streams, or different host threads
+ * without ordering between them - race on it and corrupt each other's result.  Issue them on one
+ * stream, or order them with events.
+ *
+ * Arguments as for atts_calib_update, minus the workspace.
+ */
+#define ATTS_STATIC_MAX_TOTAL 65536
+#define ATTS_STATIC_MAX_NEW 16384
+#define ATTS_STATIC_SCRATCH_BYTES (4 * ATTS_STATIC_MAX_NEW + 4 * ATTS_STATIC_MAX_TOTAL)
+int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k,
+                             int64_t* n_out, void* cuda_stream);
 
 /*
  * Waits for `cuda_stream`, then returns in *bits (host out) the OR of the ATTS_DEV_* conditions

@@ -17,6 +17,7 @@ EXPORTS = (
     "atts_strerror", "atts_version", "atts_score_workspace_bytes", "atts_score_logprob",
     "atts_conformal_rank", "atts_classify", "atts_calib_workspace_bytes", "atts_calib_update",
     "atts_last_device_status", "atts_profile_begin", "atts_profile_end",
+    "atts_calib_update_static",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -58,6 +59,7 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.atts_calib_update.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
                                       c_size_t, c_void_p]
     lib.atts_last_device_status.argtypes = [c_void_p, POINTER(c_uint32)]
+    lib.atts_calib_update_static.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p]
     lib.atts_profile_begin.argtypes = [c_int]
     lib.atts_profile_end.argtypes = [POINTER(ctypes.c_float), c_int, POINTER(c_int)]
     for name in EXPORTS[2:]:
@@ -132,6 +134,22 @@ def calib_update(calib, n: int, new_scores, workspace) -> int:
     _check(load().atts_calib_update(_ptr(calib), n, calib.numel(), _ptr(new_scores), k, ctypes.byref(n_out),
                                     _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
                                     _stream()), "atts_calib_update")
+    return n_out.value
+
+
+STATIC_MAX_TOTAL, STATIC_MAX_NEW = 65536, 16384
+
+
+def calib_update_static(calib, n: int, new_scores) -> int:
+    """Same as :func:`calib_update` without a workspace, for callers that cannot allocate device memory (an engine
+    plug-in left with no free HBM, a loop that must not pay cudaMalloc's device-wide synchronisation): the scratch is
+    a fixed array inside the library, so n + k <= STATIC_MAX_TOTAL and k <= STATIC_MAX_NEW (status 10 otherwise).
+    All calls on a device share that array: keep them on one stream or order them, overlapping calls race.
+    Make the first call on a device at start-up (it looks up the array's address). Returns n + k."""
+    n_out = c_int64(0)
+    k = 0 if new_scores is None else new_scores.numel()
+    _check(load().atts_calib_update_static(_ptr(calib), n, calib.numel(), _ptr(new_scores), k, ctypes.byref(n_out),
+                                           _stream()), "atts_calib_update_static")
     return n_out.value
 
 

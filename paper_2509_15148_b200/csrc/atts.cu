@@ -112,6 +112,33 @@ static int encode_2d(const DeviceInfo* di, CUtensorMap* map, const void* base, i
   return r == CUDA_SUCCESS ? ATTS_OK : ATTS_ERR_CUDA;
 }
 
+// Built-in scratch of atts_calib_update_static: [sorted new keys: ATTS_STATIC_MAX_NEW u32]
+// [merged copy: ATTS_STATIC_MAX_TOTAL f32].  In host code this name is only a handle for
+// cudaGetSymbolAddress; the device address it yields is what kernels are given.
+static __device__ __align__(256) unsigned char g_static_scratch[ATTS_STATIC_SCRATCH_BYTES];
+static unsigned char* g_static_scratch_addr[64] = {};
+static std::mutex g_static_mu;
+
+// Device address of the built-in scratch on the current device, looked up once per device.
+static int static_scratch(unsigned char** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return ATTS_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_scratch_addr[dev];
+  return ATTS_OK;
+}
+
 }  // namespace atts
 
 using namespace atts;
@@ -130,6 +157,8 @@ const char* atts_strerror(int status) {
     case ATTS_ERR_ARCH: return "the current device is not sm_100 (no fallback path exists)";
     case ATTS_ERR_CUDA: return "a CUDA call failed (no usable device?)";
     case ATTS_ERR_TIMEOUT: return "a bounded wait on the device expired";
+    case ATTS_ERR_SCRATCH_LIMIT:
+      return "sizes exceed the built-in scratch of the allocation-free entry point (n + k <= 65536, k <= 16384)";
     default: return "unknown status";
   }
 }
@@ -289,6 +318,40 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
       return ATTS_ERR_CUDA;
     }
     cur = total;
+  }
+  return ATTS_OK;
+}
+
+int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
+                             void* cuda_stream) {
+  if (n < 0 || k < 0 || cap < 0 || cap >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  if (n + k > cap) return ATTS_ERR_CAPACITY;
+  if (n + k > ATTS_STATIC_MAX_TOTAL || k > ATTS_STATIC_MAX_NEW) return ATTS_ERR_SCRATCH_LIMIT;
+  if ((cap > 0 && !calib) || (k > 0 && !new_scores)) return ATTS_ERR_NULL;
+  if (!aligned(calib, 4) || !aligned(new_scores, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  unsigned char* scratch = nullptr;
+  if ((st = static_scratch(&scratch)) != ATTS_OK) return st;
+  if (n_out) *n_out = n + k;
+  if (k == 0) return ATTS_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t* sorted_keys = reinterpret_cast<uint32_t*>(scratch);
+  float* merged = reinterpret_cast<float*>(scratch + 4 * ATTS_STATIC_MAX_NEW);
+  const int kc = (int)k;
+  int sort_blocks = (kc + 7) / 8;
+  if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
+  sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)kc * 4, stream>>>(new_scores, kc, sorted_keys);
+  if ((st = launch_status()) != ATTS_OK) return st;
+  const int64_t total = n + k;
+  int merge_blocks = (int)((total + kMergeThreads - 1) / kMergeThreads);
+  if (merge_blocks > di->sm_count * 4) merge_blocks = di->sm_count * 4;
+  merge_kernel<<<merge_blocks, kMergeThreads, (size_t)kc * 4, stream>>>(calib, (int)n, sorted_keys, kc, merged);
+  if ((st = launch_status()) != ATTS_OK) return st;
+  if (cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
   }
   return ATTS_OK;
 }

@@ -28,11 +28,11 @@ def test_header_symbols_are_exported():
 def test_strerror_and_version():
     assert binding.version() >= 100
     seen = set()
-    for code in range(0, 10):
+    for code in range(0, 11):
         s = binding.strerror(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 10
+    assert len(seen) == 11
     assert binding.strerror(1234) == "unknown status"
 
 
