@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 
 from paper_2509_15148_b200 import inputs  # noqa: E402
 
-WORKLOAD = "32b"
+WORKLOAD = "32b"   # the bench line's workload; --workload picks another shape for profiling runs
 ALPHA = 0.1
 METRIC = "draft tokens scored/s"
 UNIT = "tokens/s"
@@ -134,7 +134,7 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import atts_oracle as orc
-    c = inputs.CONFIGS[WORKLOAD]
+    c = inputs.CONFIGS[args.workload]
     N, T, d, V, n0 = c["N"], c["T"], c["d"], c["V"], c["n"]
     rows = args.oracle_rows
     Wb = inputs.lm_head(inputs.BASE_SEED, V, d)
@@ -247,7 +247,7 @@ def run_ours(args):
     binding.load()
     peaks, peak_kind = measured_peaks()
 
-    c = inputs.CONFIGS[WORKLOAD]
+    c = inputs.CONFIGS[args.workload]
     N, T, d, V, n0 = c["N"], c["T"], c["d"], c["V"], c["n"]
     M = N * T
     K, Wm = args.steps, args.warmup
@@ -376,10 +376,10 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": f"32B-target shape: N={N} samples x T={T} tokens per GPU, d={d}, V={V}, online calibration "
+        "config": {"workload": f"{args.workload.upper()}-target shape: N={N} samples x T={T} tokens per GPU, d={d}, V={V}, online calibration "
                                f"n={n0} growing by {N * world} per step, alpha={ALPHA}",
                    "step": "score_logprob + conformal_rank + classify + calib_update",
-                   "l2": "inputs larger than L2 (H 671 MB, W 1557 MB per step), no flush needed",
+                   "l2": f"inputs larger than L2 (H {M * d * 2 / 1e6:.0f} MB, W {V * d * 2 / 1e6:.0f} MB per step), no flush needed",
                    "parallelism": f"dp{world}: samples sharded, W replicated, all-gather of {N} scores per rank"
                    if world > 1 else "single GPU"},
         "clocks": clocks,
@@ -390,7 +390,8 @@ def run_ours(args):
                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": achieved / peaks["bf16_tflops_sustained"], "peak_kind": f"{peak_kind}, sustained bf16 GEMM "
                      "(kernel timed inside a long step)", "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
-                     "kernel_ms": k1_avg, "flops_per_launch": flops, "traffic": k1_traffic_bytes()},
+                     "kernel_ms": k1_avg, "flops_per_launch": flops,
+                     "traffic": k1_traffic_bytes() if args.workload == WORKLOAD else None},
         "stage_counts_last_step": stage_counts_last, "calib_n_end": state["n"],
     }
     if rank == 0 and world == 1:
@@ -421,6 +422,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--oracle-rows", type=int, default=256, help="token rows the CPU oracle scores per step")
+    ap.add_argument("--workload", default=WORKLOAD, choices=sorted(inputs.CONFIGS),
+                    help="shape to run (default: the bench line's workload; others are for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-conformal", action="store_true")
     args = ap.parse_args()
