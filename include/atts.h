@@ -129,6 +129,21 @@ int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sort
 int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, uint8_t* stage,
                   uint32_t* stage_counts, void* cuda_stream);
 
+/*
+ * atts_conformal_rank and atts_classify for up to four rejection rates in one launch (the
+ * conformal-only workload thresholds the same p-values at several alpha).  Outputs are byte for
+ * byte those of one atts_conformal_rank call followed by n_alpha atts_classify calls.
+ *
+ *   alphas        host [n_alpha] double, each in (0, 1); 1 <= n_alpha <= 4
+ *   numer, pvalue      as atts_conformal_rank
+ *   stage         dev  [n_alpha][Nc] uint8 out (row a holds the stages at alphas[a]), 16-byte
+ *                      aligned; with n_alpha > 1, Nc must be a multiple of 16 so that every row is
+ *   stage_counts  dev  [n_alpha][3] uint32 out, overwritten; may be NULL
+ */
+int atts_rank_classify(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
+                       const double* alphas, int32_t n_alpha, uint32_t* numer, float* pvalue,
+                       uint8_t* stage, uint32_t* stage_counts, void* cuda_stream);
+
 /* Bytes of workspace atts_calib_update needs to insert k scores into a buffer holding n. */
 int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes);
 

@@ -17,7 +17,7 @@ EXPORTS = (
     "atts_strerror", "atts_version", "atts_score_workspace_bytes", "atts_score_logprob",
     "atts_conformal_rank", "atts_classify", "atts_calib_workspace_bytes", "atts_calib_update",
     "atts_last_device_status", "atts_profile_begin", "atts_profile_end",
-    "atts_calib_update_static",
+    "atts_calib_update_static", "atts_rank_classify",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -55,6 +55,8 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
                                        c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.atts_conformal_rank.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_void_p]
     lib.atts_classify.argtypes = [c_void_p, c_int64, c_int64, c_double, c_void_p, c_void_p, c_void_p]
+    lib.atts_rank_classify.argtypes = [c_void_p, c_int64, c_void_p, c_int64, POINTER(c_double), c_int32, c_void_p, c_void_p,
+                                       c_void_p, c_void_p, c_void_p]
     lib.atts_calib_workspace_bytes.argtypes = [c_int64, c_int64, POINTER(c_size_t)]
     lib.atts_calib_update.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
                                       c_size_t, c_void_p]
@@ -118,6 +120,13 @@ def classify(numer, n: int, alpha: float, stage, stage_counts=None) -> None:
     """numer [Nc] u32 -> stage [Nc] u8, stage_counts [3] u32 (int32 storage) or None."""
     _check(load().atts_classify(_ptr(numer), numer.numel(), n, float(alpha), _ptr(stage), _ptr(stage_counts),
                                 _stream()), "atts_classify")
+
+
+def rank_classify(scores, calib_sorted, n: int, alphas, numer, pvalue, stage, stage_counts=None) -> None:
+    """Rank and threshold at up to four alphas in one launch: stage [len(alphas), Nc] u8, stage_counts [len(alphas), 3]."""
+    arr = (c_double * len(alphas))(*[float(a) for a in alphas])
+    _check(load().atts_rank_classify(_ptr(scores), scores.numel(), _ptr(calib_sorted), n, arr, len(alphas), _ptr(numer),
+                                     _ptr(pvalue), _ptr(stage), _ptr(stage_counts), _stream()), "atts_rank_classify")
 
 
 def calib_workspace_bytes(n: int, k: int) -> int:

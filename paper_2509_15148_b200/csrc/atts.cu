@@ -53,7 +53,6 @@ static int device_info(const DeviceInfo** out) {
       di.encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
       ok = ok && cudaFuncSetAttribute(lmhead_lse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kScoreSmemBytes) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(rank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kSortMaxK * 4) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -224,6 +223,35 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
   return ATTS_OK;
 }
 
+// Shared launcher of the rank kernel, with or without the fused thresholding.
+static int launch_rank(const DeviceInfo* di, const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
+                       uint32_t* numer, float* pvalue, int n_alpha, const FusedClassify& fc, cudaStream_t stream) {
+  // Table: the whole buffer when it has at most 8191 entries, else every 2^L-th entry.  Few candidates do
+  // not repay a large strided table fill, so they get a smaller one.
+  const int64_t max_slots = (Nc >= (1 << 16) ? (1 << kRankMaxTableLog2) : (1 << 10)) - 1;
+  int L = 0;
+  if (n > (1 << kRankMaxTableLog2) - 1)
+    while (((n + (1ll << L) - 1) >> L) > max_slots) ++L;
+  const int ns = (int)((n + (1ll << L) - 1) >> L);
+  int P = 1;
+  while ((1 << P) - 1 < ns) ++P;
+  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
+  int64_t blocks = (Nc + per_block - 1) / per_block;
+  // one block per SM when the table is filled by strided loads (the fill is paid per block), two otherwise
+  const int64_t max_blocks = (int64_t)di->sm_count * (L == 0 ? 2 : 1);
+  if (blocks > max_blocks) blocks = max_blocks;
+  const dim3 grid((unsigned)blocks), block(kRankThreads);
+  const size_t smem = (size_t)4 << P;
+  switch (n_alpha) {
+    case 0: rank_kernel<0><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;
+    case 1: rank_kernel<1><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;
+    case 2: rank_kernel<2><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;
+    case 3: rank_kernel<3><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;
+    default: rank_kernel<4><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;
+  }
+  return launch_status();
+}
+
 int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n, uint32_t* numer,
                         float* pvalue, void* cuda_stream) {
   if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
@@ -234,19 +262,38 @@ int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sort
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
   if (Nc == 0) return ATTS_OK;
-  // Splitter level: whole buffer in shared memory up to 8192 entries, else every 2^L-th entry with
-  // at most 2048 splitters.
-  int L = 0;
-  if (n > 8192)
-    while (((n + (1ll << L) - 1) >> L) > 2048) ++L;
-  const int ns = (int)((n + (1ll << L) - 1) >> L);
-  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
-  int64_t blocks = (Nc + per_block - 1) / per_block;
-  const int64_t max_blocks = (int64_t)di->sm_count * 8;
-  if (blocks > max_blocks) blocks = max_blocks;
-  rank_kernel<<<(unsigned)blocks, kRankThreads, (size_t)ns * 4, static_cast<cudaStream_t>(cuda_stream)>>>(
-      scores, Nc, calib_sorted, (int)n, ns, L, numer, pvalue);
-  return launch_status();
+  return launch_rank(di, scores, Nc, calib_sorted, n, numer, pvalue, 0, FusedClassify{}, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int atts_rank_classify(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n, const double* alphas,
+                       int32_t n_alpha, uint32_t* numer, float* pvalue, uint8_t* stage, uint32_t* stage_counts,
+                       void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  if (n_alpha < 1 || n_alpha > kMaxAlphas) return ATTS_ERR_ARG;
+  if (!alphas) return ATTS_ERR_NULL;
+  for (int a = 0; a < n_alpha; ++a)
+    if (!(alphas[a] > 0.0 && alphas[a] < 1.0)) return ATTS_ERR_ARG;
+  if (Nc > 0 && (!scores || !numer || !stage)) return ATTS_ERR_NULL;
+  if (n > 0 && !calib_sorted) return ATTS_ERR_NULL;
+  if (!aligned(scores, 16) || !aligned(numer, 16) || !aligned(pvalue, 16) || !aligned(calib_sorted, 4) ||
+      !aligned(stage, 16) || !aligned(stage_counts, 4) || (n_alpha > 1 && Nc % 16 != 0))
+    return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (stage_counts && cudaMemsetAsync(stage_counts, 0, (size_t)n_alpha * 3 * sizeof(uint32_t), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  if (Nc == 0) return ATTS_OK;
+  FusedClassify fc{};
+  for (int a = 0; a < n_alpha; ++a) {
+    fc.k_alpha[a] = (uint32_t)floor(alphas[a] * (double)(n + 1));
+    fc.stage[a] = stage + (size_t)a * Nc;
+  }
+  fc.counts = stage_counts;
+  return launch_rank(di, scores, Nc, calib_sorted, n, numer, pvalue, n_alpha, fc, stream);
 }
 
 int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, uint8_t* stage, uint32_t* stage_counts,
@@ -300,13 +347,14 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
   const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
   uint32_t* sorted_keys = static_cast<uint32_t*>(workspace);
   float* merged = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up((size_t)kk * 4, 256));
-  // Batches larger than one sort launch handles are inserted slice by slice.
+  // Sort the new keys, merge into the workspace, copy back.  Batches larger than one sort launch handles are
+  // inserted slice by slice.
   int64_t cur = n;
   for (int64_t off = 0; off < k; off += kSortMaxK) {
     const int kc = (int)((k - off) < kSortMaxK ? (k - off) : kSortMaxK);
     int sort_blocks = (kc + 7) / 8;
     if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
-    sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)kc * 4, stream>>>(new_scores + off, kc, sorted_keys);
+    sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)((kc + 127) & ~127) * 4, stream>>>(new_scores + off, kc, sorted_keys);
     if ((st = launch_status()) != ATTS_OK) return st;
     int64_t total = cur + kc;
     int merge_blocks = (int)((total + kMergeThreads - 1) / kMergeThreads);
@@ -342,7 +390,7 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
   const int kc = (int)k;
   int sort_blocks = (kc + 7) / 8;
   if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
-  sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)kc * 4, stream>>>(new_scores, kc, sorted_keys);
+  sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)((kc + 127) & ~127) * 4, stream>>>(new_scores, kc, sorted_keys);
   if ((st = launch_status()) != ATTS_OK) return st;
   const int64_t total = n + k;
   int merge_blocks = (int)((total + kMergeThreads - 1) / kMergeThreads);

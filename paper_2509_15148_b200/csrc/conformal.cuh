@@ -29,79 +29,159 @@ __device__ __forceinline__ uint32_t bits_of_key(uint32_t k) {
 //
 // lower_bound = number of leading entries with calib[i] < s.  With NaNs sorted last the predicate
 // calib[i] < s is true on a prefix and false after it, NaNs included, so NaN calibration entries
-// count as ">= s".  The search is two-level: a block first copies `ns` evenly spaced splitters
-// sp[t] = calib[t << L] into shared memory, a thread finds the splitter interval there and
-// finishes in the (L2-resident) buffer over at most 2^L entries.  With L == 0 the whole buffer is
-// in shared memory and the second level is skipped.
+// count as ">= s".  The search is two-level and branch-free.  A block first copies the splitters
+// sp[t] = calib[t << L], t < ns, into a shared table laid out as an implicit search tree in
+// breadth-first order (2^P - 1 nodes; node b at depth l holds the splitter of sorted rank
+// (2q + 1) * 2^(P-1-l) - 1, q = b - 2^l; ranks >= ns hold NaN, which never compares "less").
+// Descending it takes exactly P steps, and nodes of one depth are contiguous, so the lanes of a
+// warp spread over the banks (a sorted table probed at rank +- step puts every lane in one bank).
+// The leaf reached gives the number of splitters below the score; the entries below it among the
+// 2^L - 1 buffer entries that follow the last such splitter are counted in exactly L steps of
+// (L2-resident) global loads.  With L == 0 the table is the whole buffer.  A thread carries four
+// scores through every step together, so their loads overlap.
 // ---------------------------------------------------------------------------------------------
-constexpr int kRankThreads = 256;
+constexpr int kRankThreads = 1024;
 constexpr int kRankPerThread = 4;
+constexpr int kRankMaxTableLog2 = 13;  // table of at most 8191 splitters (32 KB)
 
-__device__ __forceinline__ uint32_t rank_one(float s, const float* __restrict__ sp, int ns, int L,
-                                             const float* __restrict__ calib, int n) {
-  if (s != s) return 0u;  // NaN candidate: no score
-  // t = number of splitters < s
-  int lo = 0, len = ns;
-  while (len > 0) {
-    int half = len >> 1;
-    bool less = sp[lo + half] < s;
-    lo = less ? lo + half + 1 : lo;
-    len = less ? len - half - 1 : half;
+__device__ __forceinline__ void rank_four(const float (&s)[4], const float* __restrict__ sp, int P, int L,
+                                          const float* __restrict__ calib, int n, uint32_t (&numer)[4]) {
+  int cnt[4] = {1, 1, 1, 1};  // breadth-first node number, from the root
+  for (int depth = 0; depth < P; ++depth) {
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = sp[cnt[e] - 1];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) cnt[e] = 2 * cnt[e] + ((v[e] < s[e]) ? 1 : 0);
   }
-  int below;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) cnt[e] -= 1 << P;  // leaf number = splitters below the score
+  int below[4];
   if (L == 0) {
-    below = lo;
-  } else if (lo == 0) {
-    below = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) below[e] = cnt[e];
   } else {
-    // calib[(lo-1) << L] < s and (if it exists) calib[lo << L] >= s
-    int a = ((lo - 1) << L) + 1;
-    int b = min(lo << L, n);
-    int len2 = b - a;
-    while (len2 > 0) {
-      int half = len2 >> 1;
-      bool less = __ldg(calib + a + half) < s;
-      a = less ? a + half + 1 : a;
-      len2 = less ? len2 - half - 1 : half;
+    // calib[(cnt-1) << L] < s and, if it exists, calib[cnt << L] >= s: the answer is base + (number of
+    // entries below s among calib[base .. base + 2^L - 2]) with base = ((cnt-1) << L) + 1.
+    int base[4], pos[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) base[e] = cnt[e] ? ((cnt[e] - 1) << L) + 1 : n;
+    for (int step = 1 << (L - 1); step > 0; step >>= 1) {
+      float v[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int idx = base[e] + pos[e] + step - 1;
+        v[e] = idx < n ? __ldg(calib + idx) : __uint_as_float(0x7FC00000u);
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) pos[e] += (v[e] < s[e]) ? step : 0;
     }
-    below = a;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) below[e] = cnt[e] ? base[e] + pos[e] : 0;
   }
-  return (uint32_t)(n - below) + 1u;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) numer[e] = (s[e] != s[e]) ? 0u : (uint32_t)(n - below[e]) + 1u;  // NaN: no score
 }
 
+// Stage of a sample (accept iff p > alpha  <=>  numer > k_alpha): 1 no score, 2 accepted, 3 target takes over.
+__device__ __forceinline__ uint32_t stage_of(uint32_t numer, uint32_t k_alpha) {
+  return numer == 0u ? 1u : (numer <= k_alpha ? 3u : 2u);
+}
+
+constexpr int kMaxAlphas = 4;
+// Optional thresholding fused into the rank kernel: for each of NA rejection rates the stage bytes and the
+// three stage counts, exactly what classify_kernel would produce from the numerators.
+struct FusedClassify {
+  uint32_t k_alpha[kMaxAlphas];
+  uint8_t* stage[kMaxAlphas];
+  uint32_t* counts;  // [NA][3] or nullptr
+};
+
+template <int NA>
 __global__ void __launch_bounds__(kRankThreads)
 rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restrict__ calib, int n,
-            int ns, int L, uint32_t* __restrict__ numer, float* __restrict__ pvalue) {
+            int ns, int P, int L, uint32_t* __restrict__ numer, float* __restrict__ pvalue,
+            const FusedClassify fc) {
   extern __shared__ float sp[];
-  for (int t = threadIdx.x; t < ns; t += kRankThreads) sp[t] = __ldg(calib + ((int64_t)t << L));
+  uint32_t c1[NA > 0 ? NA : 1] = {}, c3[NA > 0 ? NA : 1] = {}, seen = 0;
+  const int slots = (1 << P) - 1;
+  for (int t = threadIdx.x; t < slots; t += kRankThreads) {
+    const int b = t + 1;                       // node number
+    const int depth = 31 - __clz(b);
+    const int q = b - (1 << depth);
+    const int rank = ((2 * q + 1) << (P - 1 - depth)) - 1;
+    sp[t] = rank < ns ? __ldg(calib + ((int64_t)rank << L)) : __uint_as_float(0x7FC00000u);
+  }
   __syncthreads();
   const float denom = (float)(n + 1);
+  const float qnan = __uint_as_float(0x7FC00000u);
   const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
   for (int64_t base = (int64_t)blockIdx.x * per_block; base < Nc; base += (int64_t)gridDim.x * per_block) {
-    int64_t j = base + (int64_t)threadIdx.x * kRankPerThread;
-    if (j + kRankPerThread <= Nc) {
-      float4 s4 = *reinterpret_cast<const float4*>(scores + j);
-      uint4 r;
-      r.x = rank_one(s4.x, sp, ns, L, calib, n);
-      r.y = rank_one(s4.y, sp, ns, L, calib, n);
-      r.z = rank_one(s4.z, sp, ns, L, calib, n);
-      r.w = rank_one(s4.w, sp, ns, L, calib, n);
-      *reinterpret_cast<uint4*>(numer + j) = r;
-      if (pvalue) {
-        const float qnan = __uint_as_float(0x7FC00000u);
-        float4 p;
-        p.x = r.x ? __fdiv_rn((float)r.x, denom) : qnan;
-        p.y = r.y ? __fdiv_rn((float)r.y, denom) : qnan;
-        p.z = r.z ? __fdiv_rn((float)r.z, denom) : qnan;
-        p.w = r.w ? __fdiv_rn((float)r.w, denom) : qnan;
-        *reinterpret_cast<float4*>(pvalue + j) = p;
-      }
+    const int64_t j = base + (int64_t)threadIdx.x * kRankPerThread;
+    if (j >= Nc) continue;
+    float s[4];
+    uint32_t r[4];
+    const bool full = j + kRankPerThread <= Nc;
+    if (full) {
+      const float4 s4 = *reinterpret_cast<const float4*>(scores + j);
+      s[0] = s4.x; s[1] = s4.y; s[2] = s4.z; s[3] = s4.w;
     } else {
-      for (int e = 0; e < kRankPerThread && j + e < Nc; ++e) {
-        uint32_t r = rank_one(scores[j + e], sp, ns, L, calib, n);
-        numer[j + e] = r;
-        if (pvalue) pvalue[j + e] = r ? __fdiv_rn((float)r, denom) : __uint_as_float(0x7FC00000u);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
+    }
+    rank_four(s, sp, P, L, calib, n, r);
+    float p[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) p[e] = r[e] ? __fdiv_rn((float)r[e], denom) : qnan;
+    if (full) {
+      *reinterpret_cast<uint4*>(numer + j) = make_uint4(r[0], r[1], r[2], r[3]);
+      if (pvalue) *reinterpret_cast<float4*>(pvalue + j) = make_float4(p[0], p[1], p[2], p[3]);
+    } else {
+      for (int e = 0; e < 4 && j + e < Nc; ++e) {
+        numer[j + e] = r[e];
+        if (pvalue) pvalue[j + e] = p[e];
       }
+    }
+    if (NA > 0) {
+      const int valid = full ? 4 : (int)(Nc - j);
+      seen += (uint32_t)valid;
+#pragma unroll
+      for (int a = 0; a < NA; ++a) {
+        uint32_t st[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          st[e] = stage_of(r[e], fc.k_alpha[a]);
+          c1[a] += (e < valid) && (st[e] == 1u);
+          c3[a] += (e < valid) && (st[e] == 3u);
+        }
+        if (full) {
+          *reinterpret_cast<uint32_t*>(fc.stage[a] + j) = st[0] | (st[1] << 8) | (st[2] << 16) | (st[3] << 24);
+        } else {
+          for (int e = 0; e < valid; ++e) fc.stage[a][j + e] = (uint8_t)st[e];
+        }
+      }
+    }
+  }
+  if (NA > 0 && fc.counts != nullptr) {
+    __shared__ uint32_t sh[kMaxAlphas][3][kRankThreads / 32];
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+      uint32_t v1 = c1[a], v3 = c3[a], v2 = seen - c1[a] - c3[a];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, o);
+        v2 += __shfl_xor_sync(0xFFFFFFFFu, v2, o);
+        v3 += __shfl_xor_sync(0xFFFFFFFFu, v3, o);
+      }
+      if (l == 0) { sh[a][0][w] = v1; sh[a][1][w] = v2; sh[a][2][w] = v3; }
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < NA * 3) {
+      const int a = threadIdx.x / 3, i = threadIdx.x % 3;
+      uint32_t t = 0;
+      for (int q = 0; q < kRankThreads / 32; ++q) t += sh[a][i][q];
+      if (t) atomicAdd(fc.counts + threadIdx.x, t);
     }
   }
 }
@@ -111,10 +191,6 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
 // ---------------------------------------------------------------------------------------------
 constexpr int kClassifyThreads = 256;
 constexpr int kClassifyPerThread = 16;
-
-__device__ __forceinline__ uint32_t stage_of(uint32_t numer, uint32_t k_alpha) {
-  return numer == 0u ? 1u : (numer <= k_alpha ? 3u : 2u);
-}
 
 __global__ void __launch_bounds__(kClassifyThreads)
 classify_kernel(const uint32_t* __restrict__ numer, int64_t Nc, uint32_t k_alpha,
@@ -166,30 +242,47 @@ classify_kernel(const uint32_t* __restrict__ numer, int64_t Nc, uint32_t k_alpha
 }
 
 // ---------------------------------------------------------------------------------------------
-// K5  sort of the new calibration scores by all-pairs ranking.  One warp per element: its lanes
-// stride over all k keys (held in shared memory) and count those that precede it; equal keys keep
-// their input order, so every element gets its own slot.  k is at most kSortMaxK per launch.
+// K5  sort of the new calibration scores by all-pairs ranking, spread over the whole GPU.  Every block
+// holds all k keys in shared memory (padded to a multiple of 128 with a key above every canonical key);
+// one warp per element counts, four keys per 128-bit load, the keys below it and the keys not above it.
+// If only the element itself is equal to it, the first count is its slot; otherwise (ties, rare) the
+// warp also counts the equal keys that come before it in the input, so every element gets its own slot.
+// k is at most kSortMaxK per launch.
 // ---------------------------------------------------------------------------------------------
 constexpr int kSortMaxK = 16384;
 constexpr int kSortThreads = 256;
 
 __global__ void __launch_bounds__(kSortThreads)
 sort_new_kernel(const float* __restrict__ new_scores, int k, uint32_t* __restrict__ sorted_keys) {
-  extern __shared__ uint32_t keys[];
-  for (int t = threadIdx.x; t < k; t += kSortThreads) keys[t] = key_of_bits(canonical_bits(new_scores[t]));
+  extern __shared__ __align__(16) uint32_t keys[];
+  const int kpad = (k + 127) & ~127;
+  for (int t = threadIdx.x; t < kpad; t += kSortThreads)
+    keys[t] = t < k ? key_of_bits(canonical_bits(new_scores[t])) : 0xFFFFFFFFu;
   __syncthreads();
   const int warps = kSortThreads / 32;
   const int lane = threadIdx.x & 31;
   for (int j = blockIdx.x * warps + (threadIdx.x >> 5); j < k; j += gridDim.x * warps) {
     const uint32_t kj = keys[j];
-    int cnt = 0;
-    for (int i = lane; i < k; i += 32) {
-      uint32_t ki = keys[i];
-      cnt += (ki < kj) || (ki == kj && i < j);
+    int lt = 0, le = 0;
+    for (int i = lane * 4; i < kpad; i += 128) {
+      const uint4 q = *reinterpret_cast<const uint4*>(keys + i);
+      lt += (q.x < kj) + (q.y < kj) + (q.z < kj) + (q.w < kj);
+      le += (q.x <= kj) + (q.y <= kj) + (q.z <= kj) + (q.w <= kj);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
-    if (lane == 0) sorted_keys[cnt] = kj;
+    for (int o = 16; o > 0; o >>= 1) {
+      lt += __shfl_xor_sync(0xFFFFFFFFu, lt, o);
+      le += __shfl_xor_sync(0xFFFFFFFFu, le, o);
+    }
+    int slot = lt;
+    if (le - lt > 1) {  // equal keys: input order decides
+      int before = 0;
+      for (int i = lane; i < j; i += 32) before += keys[i] == kj;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, o);
+      slot += before;
+    }
+    if (lane == 0) sorted_keys[slot] = kj;
   }
 }
 

@@ -111,7 +111,8 @@ def test_classify_boundary_cases_and_no_counts():
 
 
 @pytest.mark.parametrize("n,k", [(0, 1), (0, 300), (1, 1), (256, 8), (4096, 64), (1000, 4097), (65536, 4096),
-                                  (323584, 4096), (5000, 16384), (100, 40000), (7, 0)])
+                                  (323584, 4096), (5000, 16384), (100, 40000), (7, 0),
+                                  (602112, 4096), (602113, 4096), (700000, 100), (20, 16385)])
 def test_calib_update_bit_exact(n, k):
     calib = np.sort(inputs.lognormal_scores(300 + n, n))
     new = inputs.lognormal_scores(400 + k, k)
@@ -120,6 +121,31 @@ def test_calib_update_bit_exact(n, k):
     want = orc.calib_update(calib, new)
     assert np.array_equal(f32_bits(buf[:n2]), f32_bits(want))
     assert np.all(f32_bits(buf[n2:]) == 0xFFFFFFFF)     # nothing written past the new fill
+
+
+@pytest.mark.parametrize("Nc,n,alphas", [(16, 9, (0.1,)), (4096 + 16, 255, (0.05, 0.1)), (1 << 20, 65536, (0.05, 0.1, 0.2)),
+                                         (100000 - 100000 % 16, 327680, (0.05, 0.1, 0.2, 0.4)), (37, 500, (0.25,))])
+def test_fused_rank_classify_equals_separate_calls(Nc, n, alphas):
+    scores = inputs.lognormal_scores(500 + Nc, Nc)
+    scores[: min(Nc, 2)] = np.array([np.nan, -1.0], np.float32)[: min(Nc, 2)]
+    calib = np.sort(inputs.lognormal_scores(600 + n, n))
+    s, c = dev(scores), dev(calib)
+    numer = poison((Nc,), torch.int32)
+    p = poison((Nc,), torch.float32)
+    stage = poison((len(alphas), Nc), torch.uint8)
+    counts = poison((len(alphas), 3), torch.int32)
+    binding.rank_classify(s, c, n, alphas, numer, p, stage, counts)
+    torch.cuda.synchronize()
+    want_numer = orc.conformal_numer_sorted(scores, calib)
+    assert np.array_equal(host_u32(numer), want_numer)
+    assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, n)))
+    for a, alpha in enumerate(alphas):
+        want_stage, want_counts = orc.classify(want_numer, n, alpha)
+        assert np.array_equal(stage[a].cpu().numpy(), want_stage)
+        assert np.array_equal(host_u32(counts[a]), want_counts)
+        # and byte for byte what the two separate entry points give
+        st2, c2 = gpu_classify(host_u32(numer), n, alpha)
+        assert np.array_equal(stage[a].cpu().numpy(), st2) and np.array_equal(host_u32(counts[a]), c2)
 
 
 def test_calib_update_duplicates_and_special_values():
@@ -162,16 +188,23 @@ def test_conformal_stress_sequence_bit_exact():
     counts = poison((3,), torch.int32)
     ws = workspace(binding.calib_workspace_bytes(cap, k))
     n = n0
+    stage_f = poison((len(cfg["alphas"]), Nc), torch.uint8)
+    counts_f = poison((len(cfg["alphas"]), 3), torch.int32)
     for t in range(steps):
+        binding.rank_classify(s_dev, buf, n, cfg["alphas"], numer, p, stage_f, counts_f)
+        fused = (host_u32(numer).copy(), stage_f.cpu().numpy().copy(), host_u32(counts_f).copy())
+        numer.view(torch.uint8).fill_(0xFF)
         binding.conformal_rank(s_dev, buf, n, numer, p)
         want_numer = orc.conformal_numer_sorted(scores, calib)
         assert np.array_equal(host_u32(numer), want_numer)
         assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, n)))
-        for alpha in cfg["alphas"]:
+        assert np.array_equal(fused[0], want_numer)
+        for a, alpha in enumerate(cfg["alphas"]):
             binding.classify(numer, n, alpha, stage, counts)
             want_stage, want_counts = orc.classify(want_numer, n, alpha)
             assert np.array_equal(stage.cpu().numpy(), want_stage)
             assert np.array_equal(host_u32(counts), want_counts)
+            assert np.array_equal(fused[1][a], want_stage) and np.array_equal(fused[2][a], want_counts)
         new = inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, k)
         n = binding.calib_update(buf, n, dev(new), ws)
         calib = orc.calib_update(calib, new)

@@ -1,0 +1,83 @@
+"""GPU parity at the full sizes of the 7B-, 32B- and 70B-target shapes, in the launch configuration the
+benchmark times.  The oracle cannot score every row in float64 (up to 1e14 flop), so it scores a seeded
+sample: every row of one whole draft sample (for the per-sample score) plus rows scattered over the rest
+of the batch.  Each sampled row still spans the whole vocabulary and the whole hidden dimension."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import atts_oracle as orc
+from paper_2509_15148_b200 import binding, inputs
+from tests.gpu_util import dev, dev_bf16, f32_bits, host_u32, poison, workspace
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3
+
+
+@pytest.mark.parametrize("name,scattered", [("7b", 192), ("32b", 192), ("70b", 128)])
+def test_full_shape_sampled_rows(name, scattered):
+    c = inputs.CONFIGS[name]
+    N, T, d, V = c["N"], c["T"], c["d"], c["V"]
+    M = N * T
+    Wb = inputs.lm_head(inputs.BASE_SEED, V, d)
+    Hb = inputs.hidden(inputs.BASE_SEED + 1, M, d)
+    ids = inputs.zipf_ids(inputs.BASE_SEED + 2, M, V)
+    off = inputs.seg_offsets(N, T)
+    # directed ids on a few rows: both ends of the vocabulary and tile edges of the last tiles
+    ids[:8] = np.array([0, 255, 256, V - 1, V - 2, (V // 256) * 256 - 1, (V // 256) * 256 % V, V // 2], np.int32)
+    lp = poison((M,), torch.float32)
+    sc = poison((N,), torch.float32)
+    ws = workspace(binding.score_workspace_bytes(M, d, V, N))
+    binding.score_logprob(dev_bf16(Hb), dev_bf16(Wb), dev(ids), dev(off), lp, sc, ws)
+    assert binding.last_device_status() == 0
+    lp_h, sc_h = lp.cpu().numpy(), sc.cpu().numpy()
+    assert np.isfinite(lp_h).all() and np.isfinite(sc_h).all()
+
+    rng = np.random.default_rng(7)
+    sample = int(rng.integers(0, N))
+    rows = np.concatenate([np.arange(8), np.arange(sample * T, (sample + 1) * T),
+                           rng.choice(M, size=scattered, replace=False)])
+    rows = np.unique(rows)
+    want = orc.token_logprob(Hb[rows], Wb, ids[rows])
+    err = np.abs(lp_h[rows].astype(np.float64) - want)
+    assert err.max() <= TOL, f"{name}: max |logprob error| {err.max():.3e}"
+    srows = np.arange(sample * T, (sample + 1) * T)
+    want_score = orc.sample_score(want[np.searchsorted(rows, srows)], np.array([0, T]))[0]
+    assert abs(float(sc_h[sample]) - want_score) <= TOL
+    # properties that hold for every row: log-probs are negative and no smaller than the uniform bound minus the
+    # logit spread allows; every sample's score equals the mean of the kernel's own token log-probs
+    assert (lp_h <= 0).all()
+    means = -lp_h.astype(np.float64).reshape(N, T).mean(axis=1)
+    assert np.abs(means - sc_h).max() <= 1e-5
+
+
+def test_conformal_stress_at_maximum_buffer_size():
+    """Last step of the conformal-only workload: 2^20 candidates against n = 323,584, three alphas, insert 4,096."""
+    cfg = inputs.CONFORMAL_STRESS
+    Nc, k = cfg["Nc"], cfg["k"]
+    n = cfg["n0"] + k * (cfg["steps"] - 1)
+    scores = inputs.lognormal_scores(inputs.BASE_SEED + 1, Nc)
+    calib = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, n))
+    new = inputs.lognormal_scores(inputs.BASE_SEED + 3 + cfg["steps"] - 1, k)
+    buf = poison((n + k,), torch.float32)
+    buf[:n] = dev(calib)
+    numer = poison((Nc,), torch.int32)
+    p = poison((Nc,), torch.float32)
+    stage = poison((Nc,), torch.uint8)
+    counts = poison((3,), torch.int32)
+    binding.conformal_rank(dev(scores), buf, n, numer, p)
+    want_numer = orc.conformal_numer_sorted(scores, calib)
+    assert np.array_equal(host_u32(numer), want_numer)
+    assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, n)))
+    idx = np.random.default_rng(1).choice(Nc, size=256, replace=False)
+    assert np.array_equal(want_numer[idx], orc.conformal_numer_count(scores[idx], calib))
+    for alpha in cfg["alphas"]:
+        binding.classify(numer, n, alpha, stage, counts)
+        want_stage, want_counts = orc.classify(want_numer, n, alpha)
+        assert np.array_equal(stage.cpu().numpy(), want_stage)
+        assert np.array_equal(host_u32(counts), want_counts)
+        assert abs(want_counts[2] / Nc - alpha) < 0.01       # rejection rate tracks alpha
+    n2 = binding.calib_update(buf, n, dev(new), workspace(binding.calib_workspace_bytes(n, k)))
+    assert n2 == n + k
+    assert np.array_equal(f32_bits(buf), f32_bits(orc.calib_update(calib, new)))

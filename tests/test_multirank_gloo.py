@@ -1,0 +1,65 @@
+"""World-size-2 check (gloo, CPU) of the data-parallel host logic: sample sharding, the score
+all-gather, and that every rank ends up with the same calibration buffer as one process would."""
+import os
+import socket
+
+import numpy as np
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from oracle import atts_oracle as orc
+from paper_2509_15148_b200 import inputs, sharding
+
+
+def test_sample_range_partitions_the_batch():
+    for n in (0, 1, 7, 64, 65):
+        for world in (1, 2, 3, 8):
+            spans = [sharding.sample_range(n, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == n
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            sizes = [b - a for a, b in spans]
+            assert max(sizes) - min(sizes) <= 1
+    assert len({sharding.rank_seed(1234, r, s) for r in range(8) for s in range(3)}) == 24
+
+
+def _worker(rank: int, world: int, port: int, out_dir: str):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    calib = np.sort(inputs.lognormal_scores(50, 300))                     # replicated buffer
+    n = calib.size
+    stages = []
+    for step in range(3):
+        local = inputs.lognormal_scores(sharding.rank_seed(60 + 10 * step, rank), 16)   # this rank's 16 scores
+        numer = orc.conformal_numer_sorted(local, calib)                  # rank against the buffer as it was
+        stages.append(orc.classify(numer, n, 0.1)[0])
+        allv = sharding.all_gather_scores(torch.from_numpy(local), world, dist).numpy()
+        calib = orc.calib_update(calib, allv)                             # every rank inserts all ranks' scores
+        n = calib.size
+    np.save(os.path.join(out_dir, f"calib_{rank}.npy"), calib)
+    np.save(os.path.join(out_dir, f"stage_{rank}.npy"), np.concatenate(stages))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_keep_identical_buffers(tmp_path):
+    world = 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    bufs = [np.load(tmp_path / f"calib_{r}.npy") for r in range(world)]
+    assert np.array_equal(bufs[0].view(np.uint32), bufs[1].view(np.uint32))
+    # one process doing the same inserts in rank order gets the same buffer
+    calib = np.sort(inputs.lognormal_scores(50, 300))
+    want_stage = {r: [] for r in range(world)}
+    for step in range(3):
+        locals_ = [inputs.lognormal_scores(sharding.rank_seed(60 + 10 * step, r), 16) for r in range(world)]
+        for r in range(world):
+            want_stage[r].append(orc.classify(orc.conformal_numer_sorted(locals_[r], calib), calib.size, 0.1)[0])
+        calib = orc.calib_update(calib, np.concatenate(locals_))
+    assert calib.size == 300 + 3 * 32
+    assert np.array_equal(bufs[0].view(np.uint32), calib.view(np.uint32))
+    for r in range(world):
+        assert np.array_equal(np.load(tmp_path / f"stage_{r}.npy"), np.concatenate(want_stage[r]))
