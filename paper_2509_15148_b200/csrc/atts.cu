@@ -19,6 +19,7 @@ struct DeviceInfo {
   bool ready = false;
   int status = ATTS_OK;  // sticky result of the probe
   int sm_count = 0;
+  int pair_workers = 0;  // CTA pairs (clusters of 2) of the fused kernel that can be resident at once; 0 = unusable
   unsigned int* dev_status = nullptr;
   PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
 };
@@ -51,8 +52,29 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
            q == cudaDriverEntryPointSuccess && fn != nullptr;
       di.encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
-      ok = ok && cudaFuncSetAttribute(lmhead_lse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      kScoreSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(lmhead_lse_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      ScoreCfg<1>::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(lmhead_lse_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      ScoreCfg<2>::kSmemBytes) == cudaSuccess;
+      if (ok) {
+        // how many clusters of two CTAs fit the device at once (GPC boundaries may strand an SM)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * (unsigned)di.sm_count);
+        cfg.blockDim = dim3(kScoreThreads);
+        cfg.dynamicSmemBytes = ScoreCfg<2>::kSmemBytes;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, lmhead_lse_kernel<2>, &cfg) == cudaSuccess && clusters > 0)
+          di.pair_workers = clusters < di.sm_count / 2 ? clusters : di.sm_count / 2;
+        else
+          cudaGetLastError();
+      }
       ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kSortMaxK * 4) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -91,6 +113,22 @@ static ScoreWs score_ws(const ScorePlan& p) {
   w.total = w.logprob_off + round_up((size_t)p.M_pad * sizeof(float), 256);
   if (w.total == 0) w.total = 256;
   return w;
+}
+
+// The schedule of a scoring call.  CTA pairs keep the tensor pipe busier per clock (measured 88-97 % against
+// 81-89 %), but once H no longer fits one L2-resident panel their placement (the two CTAs of a cluster and
+// neighbouring clusters sit on adjacent SMs) multiplies DRAM traffic and, under the power cap, costs more clock
+// than it gains.  So pairs are used when all of H is one panel and their makespan (in tile times) is no longer
+// than that of single CTAs; larger batches run on single CTAs.
+static ScorePlan choose_score_plan(const DeviceInfo* di, int64_t M, int64_t d, int64_t V) {
+  const ScorePlan one = make_score_plan(M, d, V, di->sm_count, 1);
+  if (di->pair_workers <= 0 || M == 0) return one;
+  const ScorePlan two = make_score_plan(M, d, V, di->pair_workers, 2);
+  auto span = [](const ScorePlan& p, int workers) {
+    return (long long)((p.units + workers - 1) / workers) * ((p.NT + p.C - 1) / p.C);
+  };
+  const bool one_panel = two.RB <= two.Gr;
+  return (one_panel && span(two, di->pair_workers) <= span(one, di->sm_count)) ? two : one;
 }
 
 static int check_score_shape(int64_t M, int64_t d, int64_t V, int64_t S) {
@@ -171,7 +209,7 @@ int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_
   const DeviceInfo* di;
   st = device_info(&di);
   if (st != ATTS_OK) return st;
-  *bytes = score_ws(make_score_plan(M, d, V, di->sm_count)).total;
+  *bytes = score_ws(choose_score_plan(di, M, d, V)).total;
   return ATTS_OK;
 }
 
@@ -191,7 +229,7 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
   const DeviceInfo* di;
   st = device_info(&di);
   if (st != ATTS_OK) return st;
-  const ScorePlan plan = make_score_plan(M, d, V, di->sm_count);
+  const ScorePlan plan = choose_score_plan(di, M, d, V);
   const ScoreWs ws = score_ws(plan);
   if (workspace_bytes < ws.total) return ATTS_ERR_WORKSPACE;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -203,12 +241,33 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
   if (M > 0) {
     CUtensorMap map_h, map_w;
     if (encode_2d(di, &map_h, hidden_bf16, M, d, kBlockM) != ATTS_OK) return ATTS_ERR_CUDA;
-    if (encode_2d(di, &map_w, lm_head_bf16, V, d, kBlockN) != ATTS_OK) return ATTS_ERR_CUDA;
-    const int grid = plan.units < di->sm_count ? plan.units : di->sm_count;
+    if (encode_2d(di, &map_w, lm_head_bf16, V, d, kBlockN / plan.ctas) != ATTS_OK) return ATTS_ERR_CUDA;
     const bool timed = g_prof.on && g_prof.used < g_prof.cap;
     if (timed) cudaEventRecord(g_prof.ev[2 * g_prof.used], stream);
-    lmhead_lse_kernel<<<grid, kScoreThreads, kScoreSmemBytes, stream>>>(map_h, map_w, token_ids, plan, partial,
-                                                                        gathered, di->dev_status);
+    if (plan.ctas == 1) {
+      const int grid = plan.units < di->sm_count ? plan.units : di->sm_count;
+      lmhead_lse_kernel<1><<<grid, kScoreThreads, ScoreCfg<1>::kSmemBytes, stream>>>(map_h, map_w, token_ids, plan, partial,
+                                                                                     gathered, di->dev_status);
+    } else {
+      const int pairs = plan.units < di->pair_workers ? plan.units : di->pair_workers;
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(2 * (unsigned)pairs);
+      cfg.blockDim = dim3(kScoreThreads);
+      cfg.dynamicSmemBytes = ScoreCfg<2>::kSmemBytes;
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      if (cudaLaunchKernelEx(&cfg, lmhead_lse_kernel<2>, map_h, map_w, token_ids, plan, partial, gathered,
+                             di->dev_status) != cudaSuccess) {
+        cudaGetLastError();
+        return ATTS_ERR_CUDA;
+      }
+    }
     if (timed) cudaEventRecord(g_prof.ev[2 * g_prof.used++ + 1], stream);
     if ((st = launch_status()) != ATTS_OK) return st;
     lse_combine_kernel<<<(unsigned)((M + 255) / 256), 256, 0, stream>>>(partial, gathered, token_ids, (int)M, plan.M_pad,

@@ -12,32 +12,46 @@
 
 namespace atts {
 
-constexpr int kBlockM = 128;   // rows of H per tile (= TMEM lanes)
+constexpr int kBlockM = 128;   // rows of H per CTA tile (= TMEM lanes)
 constexpr int kBlockN = 256;   // vocabulary entries per tile (= TMEM columns per accumulator)
 constexpr int kBlockK = 64;    // bf16 elements per shared-memory stage row (128 bytes = swizzle span)
 constexpr int kUmmaK = 16;     // K of one tcgen05.mma (kind::f16)
-constexpr int kStages = 4;
-constexpr int kABytes = kBlockM * kBlockK * 2;
-constexpr int kBBytes = kBlockN * kBlockK * 2;
-constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kScoreThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
 constexpr int kTmemCols = 512;      // two 256-column accumulators
-constexpr int kScoreSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s: far beyond any legitimate wait
+
+// Two forms of the kernel.  CTAS = 1: every CTA computes 128 x 256 tiles on its own.  CTAS = 2: the two CTAs
+// of a cluster compute one 256 x 256 tile with tcgen05.mma.cta_group::2; each loads its own 128 rows of H and
+// its own 128 of the 256 vocabulary rows, so a CTA moves a third less data through L2 and shared memory per
+// flop, and the smaller stage leaves room for a deeper ring.
+template <int CTAS>
+struct ScoreCfg {
+  static constexpr int kRowsPerUnit = kBlockM * CTAS;          // rows of H per unit (row block)
+  static constexpr int kBRows = kBlockN / CTAS;                // vocabulary rows a CTA loads per stage
+  static constexpr int kABytes = kBlockM * kBlockK * 2;
+  static constexpr int kBBytes = kBRows * kBlockK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = CTAS == 1 ? 4 : 6;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  // Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128 * CTAS, N = 256.
+  static constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) |
+                                     ((uint32_t)(kRowsPerUnit >> 4) << 24);
+};
 
 // Static schedule of one launch.  A unit is (row block rb, vocabulary chunk c); chunk c covers the
 // tiles [c*NT/C, (c+1)*NT/C).  Units are numbered panel by panel (Gr row blocks each), chunk-major
-// inside a panel, and dealt round-robin to the CTAs, so that CTAs running at the same time share
-// vocabulary tiles in L2 while their row blocks stay L2-resident.
+// inside a panel, and dealt round-robin to the workers (CTAs, or CTA pairs), so that workers running at
+// the same time share vocabulary tiles in L2 while their row blocks stay L2-resident.
 struct ScorePlan {
   int M, V;
-  int RB;      // row blocks  = ceil(M / 128)
+  int RB;      // row blocks  = ceil(M / rows per unit)
   int NT;      // vocab tiles = ceil(V / 256)
   int KB;      // k blocks    = d / 64
   int C;       // chunks per row block (partials per row)
   int Gr;      // row blocks per panel
   int units;   // RB * C
-  int M_pad;   // RB * 128
+  int M_pad;   // RB * rows per unit
+  int ctas;    // 1 or 2: CTAs per worker
 };
 
 __host__ __device__ inline void decode_unit(const ScorePlan& p, int u, int& rb, int& c, int& nt0, int& nt1) {
@@ -52,29 +66,32 @@ __host__ __device__ inline void decode_unit(const ScorePlan& p, int u, int& rb, 
   nt1 = (int)(((long long)(c + 1) * p.NT) / p.C);
 }
 
-inline ScorePlan make_score_plan(int64_t M, int64_t d, int64_t V, int num_ctas) {
+// num_workers: CTAs (ctas == 1) or CTA pairs (ctas == 2) that run concurrently.
+inline ScorePlan make_score_plan(int64_t M, int64_t d, int64_t V, int num_workers, int ctas) {
   ScorePlan p{};
+  const int rows = kBlockM * ctas;
+  p.ctas = ctas;
   p.M = (int)M;
   p.V = (int)V;
-  p.RB = (int)((M + kBlockM - 1) / kBlockM);
+  p.RB = (int)((M + rows - 1) / rows);
   p.NT = (int)((V + kBlockN - 1) / kBlockN);
   p.KB = (int)(d / kBlockK);
-  p.M_pad = p.RB * kBlockM;
-  int cmax = p.NT < num_ctas ? p.NT : num_ctas;
+  p.M_pad = p.RB * rows;
+  int cmax = p.NT < num_workers ? p.NT : num_workers;
   if (p.RB > 0 && cmax > (1 << 30) / p.RB) cmax = (1 << 30) / p.RB;  // keep RB * C inside int
   if (cmax < 1) cmax = 1;
   long long best = -1;
   int bestC = 1;
   for (int C = 1; C <= cmax; ++C) {
-    long long waves = ((long long)p.RB * C + num_ctas - 1) / num_ctas;
+    long long waves = ((long long)p.RB * C + num_workers - 1) / num_workers;
     long long span = waves * ((p.NT + C - 1) / C);
     if (best < 0 || span < best) { best = span; bestC = C; }
   }
   p.C = bestC;
   // Panel height: about 30 MB of H per panel stays L2-resident while W streams past it (measured: larger panels
-  // thrash, DRAM reads grow 2x).  A multiple of 4, because CTAs whose index is congruent modulo Gr share a row
+  // thrash, DRAM reads grow 2x).  A multiple of 4, because workers whose index is congruent modulo Gr share a row
   // block and multiples of 4 measured 5-10 % faster than neighbouring heights.
-  long long gr = ((30ll << 20) / ((long long)kBlockM * d * 2) + 2) / 4 * 4;
+  long long gr = ((30ll << 20) / ((long long)rows * d * 2) + 2) / 4 * 4;
   if (gr < 4) gr = 4;
   if (gr > p.RB) gr = p.RB;
   p.Gr = (int)(gr < 1 ? 1 : gr);
@@ -131,6 +148,47 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap
       ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1)
       : "memory");
 }
+// ---- cluster forms (CTA pair) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address, in the cluster's shared window, of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted on the mbarrier
+// `bar_cluster_addr`, which may live in the other CTA of the pair.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t smem_dst, const CUtensorMap* tmap, uint32_t bar_cluster_addr, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T, 256 x 256 x 16 over the CTA pair (each CTA supplies 128 rows of A and 128 of B).
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// One arrival on the mbarrier at this offset in both CTAs of the pair once the MMAs issued so far have finished.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(tmap)) : "memory");
 }
@@ -163,10 +221,6 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
   d |= (uint64_t)2u << 61;                        // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 256.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBlockN >> 3) << 17) |
-                            ((uint32_t)(kBlockM >> 4) << 24);
-
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -189,19 +243,26 @@ __device__ __forceinline__ float ex2_approx(float x) {
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------
-// K1  the fused kernel.  Persistent: gridDim.x CTAs, CTA b runs units b, b + gridDim.x, ...
+// K1  the fused kernel.  Persistent: worker w (a CTA, or a CTA pair) runs units w, w + workers, ...
 //   partial[c * M_pad + row] = (max_v z, sum_v exp(z - max)) over the vocabulary chunk c
 //   gathered[row]            = z[row, token_ids[row]]   (written by the chunk that holds the id)
+// Barriers.  full[s]: stage s of the ring holds data (one per worker: with two CTAs it lives in the leader,
+// CTA 0 of the pair, and counts the bytes of both CTAs' loads).  empty[s]: the MMAs reading stage s are done
+// (one per CTA; the leader's commit reaches both).  tmem_full[a] / tmem_empty[a]: accumulator a is complete /
+// has been read by every epilogue warp of the worker (tmem_empty lives in the leader).
 // ------------------------------------------------------------------------------------------
+template <int CTAS>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                   const int32_t* __restrict__ token_ids, const ScorePlan plan,
                   float2* __restrict__ partial, float* __restrict__ gathered, unsigned int* __restrict__ dev_status) {
+  using Cfg = ScoreCfg<CTAS>;
+  constexpr int kStages = Cfg::kStages;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_al = smem_raw + (smem_base - smem_u32(smem_raw));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + kStages * kStageBytes);
-  const uint32_t bar0 = smem_base + kStages * kStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_al + kStages * Cfg::kStageBytes);
+  const uint32_t bar0 = smem_base + kStages * Cfg::kStageBytes;
   // barrier slots: full[0..S), empty[S..2S), tmem_full[2S..2S+2), tmem_empty[2S+2..2S+4)
   auto full_bar = [&](int s) { return bar0 + 8u * (uint32_t)s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (uint32_t)(kStages + s); };
@@ -212,6 +273,9 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;   // 0 = leader
+  const int worker = blockIdx.x / CTAS;
+  const int workers = gridDim.x / CTAS;
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmap_h);
@@ -222,36 +286,51 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tempty_bar(a), 4 * CTAS);
     }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 1) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)kTmemCols) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // the peer's barriers are initialised before anything signals them
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ---------------- TMA producer ----------------
+    // ---------------- TMA producer (every CTA loads its own operand halves) ----------------
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < plan.units && ok; u += gridDim.x) {
+      for (int u = worker; u < plan.units && ok; u += workers) {
         int rb, c, nt0, nt1;
         decode_unit(plan, u, rb, c, nt0, nt1);
+        const int row0 = rb * Cfg::kRowsPerUnit + (int)rank * kBlockM;
         for (int nt = nt0; nt < nt1 && ok; ++nt) {
+          const int col0 = nt * kBlockN + (int)rank * Cfg::kBRows;
           for (int kb = 0; kb < plan.KB; ++kb) {
             if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(full_bar(stage), kStageBytes);
-            const uint32_t sa = smem_base + (uint32_t)stage * kStageBytes;
-            tma_load_2d(sa, &tmap_h, full_bar(stage), kb * kBlockK, rb * kBlockM);
-            tma_load_2d(sa + kABytes, &tmap_w, full_bar(stage), kb * kBlockK, nt * kBlockN);
+            const uint32_t sa = smem_base + (uint32_t)stage * Cfg::kStageBytes;
+            if (CTAS == 1) {
+              mbar_expect_tx(full_bar(stage), Cfg::kStageBytes);
+              tma_load_2d(sa, &tmap_h, full_bar(stage), kb * kBlockK, row0);
+              tma_load_2d(sa + Cfg::kABytes, &tmap_w, full_bar(stage), kb * kBlockK, col0);
+            } else {
+              if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * Cfg::kStageBytes);
+              const uint32_t leader_full = map_to_cta(full_bar(stage), 0);
+              tma_load_2d_pair(sa, &tmap_h, leader_full, kb * kBlockK, row0);
+              tma_load_2d_pair(sa + Cfg::kABytes, &tmap_w, leader_full, kb * kBlockK, col0);
+            }
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -259,14 +338,14 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (the leader CTA issues for the pair) ----------------
+    if (lane == 0 && rank == 0) {
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < plan.units && ok; u += gridDim.x) {
+      for (int u = worker; u < plan.units && ok; u += workers) {
         int rb, c, nt0, nt1;
         decode_unit(plan, u, rb, c, nt0, nt1);
         for (int nt = nt0; nt < nt1 && ok; ++nt) {
@@ -276,19 +355,22 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
           for (int kb = 0; kb < plan.KB; ++kb) {
             if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t sa = smem_base + (uint32_t)stage * kStageBytes;
+            const uint32_t sa = smem_base + (uint32_t)stage * Cfg::kStageBytes;
             const uint64_t da = umma_smem_desc(sa);
-            const uint64_t db = umma_smem_desc(sa + kABytes);
+            const uint64_t db = umma_smem_desc(sa + Cfg::kABytes);
 #pragma unroll
             for (int k = 0; k < kBlockK / kUmmaK; ++k) {
               // 16 bf16 = 32 bytes further along K inside the swizzled row: +2 in 16-byte units
-              umma_bf16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), kIdesc, (uint32_t)((kb | k) != 0));
+              if (CTAS == 1) umma_bf16(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), Cfg::kIdesc, (uint32_t)((kb | k) != 0));
+              else umma_bf16_pair(tmem_d, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), Cfg::kIdesc, (uint32_t)((kb | k) != 0));
             }
-            umma_commit(empty_bar(stage));
+            if (CTAS == 1) umma_commit(empty_bar(stage));
+            else umma_commit_pair(empty_bar(stage));
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
           if (!ok) break;
-          umma_commit(tfull_bar(acc));
+          if (CTAS == 1) umma_commit(tfull_bar(acc));
+          else umma_commit_pair(tfull_bar(acc));
           acc ^= 1;
           if (acc == 0) acc_phase ^= 1u;
         }
@@ -296,17 +378,17 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
     }
     __syncwarp();
   } else {
-    // ---------------- epilogue: 4 warps, warp w reads TMEM lanes 32*(w%4) .. +31 ----------------
+    // ---------------- epilogue: 4 warps, warp w reads TMEM lanes 32*(w%4) .. +31 of its own CTA ----------------
     const int quarter = warp & 3;
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const float kLog2e = 1.4426950408889634f;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < plan.units && ok; u += gridDim.x) {
+    for (int u = worker; u < plan.units && ok; u += workers) {
       int rb, c, nt0, nt1;
       decode_unit(plan, u, rb, c, nt0, nt1);
-      const int row = rb * kBlockM + quarter * 32 + lane;
+      const int row = rb * Cfg::kRowsPerUnit + (int)rank * kBlockM + quarter * 32 + lane;
       const int y = (row < plan.M) ? token_ids[row] : -1;
       float m = -INFINITY, l = 0.f;
       for (int nt = nt0; nt < nt1; ++nt) {
@@ -350,7 +432,10 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (lane == 0) {
+          if (CTAS == 1) mbar_arrive(tempty_bar(acc));
+          else mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+        }
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
@@ -360,7 +445,8 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
 
   // ---------------- teardown ----------------
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // neither CTA leaves while the other may still touch its memory
+  else __syncthreads();
   if (*abort_flag) {
     // A wait expired.  Record it, give copies and MMAs still in flight time to land, then free TMEM.
     if (threadIdx.x == 0) atomicOr(dev_status, 2u);
@@ -369,7 +455,8 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
   }
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    if (CTAS == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
   }
 }
 

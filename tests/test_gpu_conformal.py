@@ -73,6 +73,28 @@ def test_rank_ties_extremes_and_special_values():
     assert np.array_equal(numer, np.arange(calib.size + 1, 1, -1, dtype=np.uint32))
 
 
+@pytest.mark.parametrize("n", [2, 4096, 8191, 8192, 70000])
+def test_rank_many_candidates_tied_clustered_and_special_data(n):
+    """Many candidates against plain, heavily tied, clustered (outliers), constant and special-valued buffers."""
+    Nc = (1 << 17) + 37
+    base = inputs.lognormal_scores(700 + n, n)
+    cases = {
+        "plain": base,
+        "ties": np.round(base, 1),
+        "outliers": np.concatenate([base[: n - 2], np.array([1e30, -1e30], np.float32)]) if n > 2 else base,
+        "constant": np.full(n, 2.5, np.float32),
+        "special": np.concatenate([base[: max(n - 5, 0)], np.array([np.inf, -np.inf, np.nan, 0.0, -0.0], np.float32)[: min(n, 5)]]),
+    }
+    scores = np.concatenate([inputs.lognormal_scores(800 + n, Nc - 8),
+                             np.array([0.0, -0.0, 2.5, np.inf, -np.inf, np.nan, 1e30, -1e30], np.float32)])
+    for name, vals in cases.items():
+        calib = orc.calib_update(np.zeros(0, np.float32), vals)
+        numer, p = gpu_rank(scores, calib)
+        assert np.array_equal(numer, orc.conformal_numer_sorted(scores, calib)), name
+        idx = np.concatenate([np.arange(Nc - 8, Nc), np.arange(0, Nc - 8, 4099)])
+        assert np.array_equal(numer[idx], orc.conformal_numer_count(scores[idx], calib)), name
+
+
 def test_rank_without_pvalue_output_and_empty_input():
     calib = np.sort(inputs.lognormal_scores(5, 300))
     scores = inputs.lognormal_scores(6, 77)
