@@ -287,6 +287,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.load()
     peaks, peak_kind = measured_peaks()
+    if args.conformal_only:
+        if rank == 0:
+            print(json.dumps({"conformal_stress": conformal_stress(torch, binding, peaks)}), flush=True)
+        return
 
     c = inputs.CONFIGS[args.workload]
     N, T, d, V, n0 = c["N"], c["T"], c["d"], c["V"], c["n"]
@@ -462,6 +466,8 @@ def main():
                     help="shape to run (default: the bench line's workload; others are for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-conformal", action="store_true")
+    ap.add_argument("--conformal-only", action="store_true",
+                    help="run only the conformal-only workload section and print it (for profiling those kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -75,6 +75,12 @@ static int device_info(const DeviceInfo** out) {
         else
           cudaGetLastError();
       }
+      const int rank_smem = 2 * (4 << kRankMaxTableLog2) + 64;  // splitter table + p-value table
+      ok = ok && cudaFuncSetAttribute(rank_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kSortMaxK * 4) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -300,7 +306,7 @@ static int launch_rank(const DeviceInfo* di, const float* scores, int64_t Nc, co
   const int64_t max_blocks = (int64_t)di->sm_count * (L == 0 ? 2 : 1);
   if (blocks > max_blocks) blocks = max_blocks;
   const dim3 grid((unsigned)blocks), block(kRankThreads);
-  const size_t smem = (size_t)4 << P;
+  const size_t smem = ((size_t)4 << P) + (L == 0 ? (size_t)4 * (n + 2) : 0);  // table (+ p-value table)
   switch (n_alpha) {
     case 0: rank_kernel<0><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;
     case 1: rank_kernel<1><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, ns, P, L, numer, pvalue, fc); break;

@@ -44,18 +44,43 @@ constexpr int kRankThreads = 1024;
 constexpr int kRankPerThread = 4;
 constexpr int kRankMaxTableLog2 = 13;  // table of at most 8191 splitters (32 KB)
 
-__device__ __forceinline__ void rank_four(const float (&s)[4], const float* __restrict__ sp, int P, int L,
-                                          const float* __restrict__ calib, int n, uint32_t (&numer)[4]) {
-  int cnt[4] = {1, 1, 1, 1};  // breadth-first node number, from the root
+// Descent of the breadth-first table, P levels, four scores at a time.  `off` is 4 * (node number): the node's
+// value sits at byte off - 4, its children at 2 * off and 2 * off + 4.  Returns the leaf number = number of
+// splitters below each score.
+template <int P>
+__device__ __forceinline__ void tree_descend(const float (&s)[4], const float* __restrict__ sp, int (&cnt)[4]) {
+  uint32_t off[4] = {4u, 4u, 4u, 4u};
+  const char* base = reinterpret_cast<const char*>(sp) - 4;
+#pragma unroll
   for (int depth = 0; depth < P; ++depth) {
     float v[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = sp[cnt[e] - 1];
+    for (int e = 0; e < 4; ++e) v[e] = *reinterpret_cast<const float*>(base + off[e]);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) cnt[e] = 2 * cnt[e] + ((v[e] < s[e]) ? 1 : 0);
+    for (int e = 0; e < 4; ++e) off[e] = 2u * off[e] + ((v[e] < s[e]) ? 4u : 0u);
   }
 #pragma unroll
-  for (int e = 0; e < 4; ++e) cnt[e] -= 1 << P;  // leaf number = splitters below the score
+  for (int e = 0; e < 4; ++e) cnt[e] = (int)(off[e] >> 2) - (1 << P);
+}
+
+__device__ __forceinline__ void rank_four(const float (&s)[4], const float* __restrict__ sp, int P, int L,
+                                          const float* __restrict__ calib, int n, uint32_t (&numer)[4]) {
+  int cnt[4];
+  switch (P) {  // the descent is unrolled for every table depth
+    case 1: tree_descend<1>(s, sp, cnt); break;
+    case 2: tree_descend<2>(s, sp, cnt); break;
+    case 3: tree_descend<3>(s, sp, cnt); break;
+    case 4: tree_descend<4>(s, sp, cnt); break;
+    case 5: tree_descend<5>(s, sp, cnt); break;
+    case 6: tree_descend<6>(s, sp, cnt); break;
+    case 7: tree_descend<7>(s, sp, cnt); break;
+    case 8: tree_descend<8>(s, sp, cnt); break;
+    case 9: tree_descend<9>(s, sp, cnt); break;
+    case 10: tree_descend<10>(s, sp, cnt); break;
+    case 11: tree_descend<11>(s, sp, cnt); break;
+    case 12: tree_descend<12>(s, sp, cnt); break;
+    default: tree_descend<13>(s, sp, cnt); break;
+  }
   int below[4];
   if (L == 0) {
 #pragma unroll
@@ -105,6 +130,13 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
   extern __shared__ float sp[];
   uint32_t c1[NA > 0 ? NA : 1] = {}, c3[NA > 0 ? NA : 1] = {}, seen = 0;
   const int slots = (1 << P) - 1;
+  // With the whole buffer in the table (L == 0) the p-values of all n + 2 possible numerators are tabulated
+  // behind it once per block (the same correctly rounded division), so a candidate costs one load, not a divide.
+  float* const ptab = sp + slots;
+  const bool tabulated = (L == 0) && pvalue != nullptr;
+  if (tabulated)
+    for (int t = threadIdx.x; t <= n + 1; t += kRankThreads)
+      ptab[t] = t ? __fdiv_rn((float)t, (float)(n + 1)) : __uint_as_float(0x7FC00000u);
   for (int t = threadIdx.x; t < slots; t += kRankThreads) {
     const int b = t + 1;                       // node number
     const int depth = 31 - __clz(b);
@@ -131,8 +163,13 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
     }
     rank_four(s, sp, P, L, calib, n, r);
     float p[4];
+    if (tabulated) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) p[e] = r[e] ? __fdiv_rn((float)r[e], denom) : qnan;
+      for (int e = 0; e < 4; ++e) p[e] = ptab[r[e]];
+    } else if (pvalue) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) p[e] = r[e] ? __fdiv_rn((float)r[e], denom) : qnan;
+    }
     if (full) {
       *reinterpret_cast<uint4*>(numer + j) = make_uint4(r[0], r[1], r[2], r[3]);
       if (pvalue) *reinterpret_cast<float4*>(pvalue + j) = make_float4(p[0], p[1], p[2], p[3]);
