@@ -184,3 +184,79 @@ def calib_update(calib_sorted: np.ndarray, new_scores: np.ndarray) -> np.ndarray
     """
     allv = np.concatenate([_canonical(calib_sorted), _canonical(new_scores)])
     return np.sort(allv, kind="stable")
+
+
+# ----------------------------------------------------------------------------------------------
+# Extensions beyond the marginal path ("next" rows): threshold form, conditional coverage, row scale.
+# ----------------------------------------------------------------------------------------------
+
+def threshold(calib_sorted: np.ndarray, alpha: float) -> np.float32:
+    """Score threshold equivalent to the rank rule: tau = the k_alpha-th largest calibration score.
+
+    numer <= k_alpha  <=>  fewer than k_alpha calibration scores are >= s  <=>  s > (k_alpha-th largest), ties
+    included; this is the quantile-threshold construction of the classic set-up (Eqs. quantile / pred_set) read
+    for the rejection side.  k_alpha = 0 (nobody can be rejected) gives +inf.
+    """
+    c = np.asarray(calib_sorted, dtype=np.float32)
+    ka = k_alpha(alpha, c.size)
+    if ka < 1:
+        return np.float32(np.inf)
+    return c[c.size - ka]
+
+
+def classify_by_threshold(scores: np.ndarray, tau: np.float32):
+    """Stage from one comparison per sample: 3 if s > tau, else 2; a NaN score is stage 1."""
+    s = np.asarray(scores, dtype=np.float32)
+    stage = np.full(s.size, STAGE_ACCEPTED, dtype=np.uint8)
+    with np.errstate(invalid="ignore"):
+        stage[s > np.float32(tau)] = STAGE_TARGET
+    stage[np.isnan(s)] = STAGE_DRAFT
+    counts = np.array([(stage == 1).sum(), (stage == 2).sum(), (stage == 3).sum()], dtype=np.uint32)
+    return stage, counts
+
+
+def conformal_numer_conditional(scores: np.ndarray, group_ids: np.ndarray, calib_groups):
+    """Conditional conformal p-value (Proposition 2; Sec. 3.2, last sentence of the p-value paragraph): a
+    candidate is ranked only against the calibration scores of its own input.
+
+    calib_groups[g] holds input g's calibration scores (any order).  Reading adopted (the appendix flips the
+    indicator and mixes denominators): the same count as the marginal form, 1 + #{calib in own group >= s},
+    over |group| + 1.  Returns (numer, denom) as uint32; a NaN candidate has numer 0.
+    """
+    s = np.asarray(scores, dtype=np.float32)
+    g = np.asarray(group_ids, dtype=np.int64)
+    numer = np.zeros(s.size, dtype=np.uint32)
+    denom = np.zeros(s.size, dtype=np.uint32)
+    for j in range(s.size):
+        c = np.asarray(calib_groups[g[j]], dtype=np.float32)
+        denom[j] = c.size + 1
+        numer[j] = conformal_numer_count(s[j:j + 1], c)[0]
+    return numer, denom
+
+
+def classify_conditional(numer: np.ndarray, denom: np.ndarray, alpha: float):
+    """Accept iff p > alpha with each candidate's own denominator: reject iff 1 <= numer <= floor(alpha * denom)."""
+    num = np.asarray(numer, dtype=np.uint32)
+    ka = np.floor(np.float64(alpha) * np.asarray(denom, dtype=np.float64)).astype(np.int64)
+    stage = np.full(num.size, STAGE_ACCEPTED, dtype=np.uint8)
+    stage[num == 0] = STAGE_DRAFT
+    stage[(num >= 1) & (num.astype(np.int64) <= ka)] = STAGE_TARGET
+    counts = np.array([(stage == 1).sum(), (stage == 2).sum(), (stage == 3).sum()], dtype=np.uint32)
+    return stage, counts
+
+
+def rms_inv(hidden_bits: np.ndarray, eps: float) -> np.ndarray:
+    """1 / sqrt(mean_k h[i, k]^2 + eps) per row, float64: the row factor of an RMS normalisation."""
+    H = bf16_bits_to_f64(hidden_bits)
+    return 1.0 / np.sqrt((H * H).mean(axis=1) + float(eps))
+
+
+def token_logprob_scaled(hidden_bits: np.ndarray, lm_head_bits: np.ndarray, token_ids: np.ndarray,
+                         row_scale: np.ndarray) -> np.ndarray:
+    """token_logprob with every row of logits multiplied by row_scale[i] before the softmax: the LM head applied
+    to an RMS-normalised hidden state, z_i = r_i * (W h_i), with the norm's gain folded into W by the caller."""
+    ids = np.asarray(token_ids, dtype=np.int64)
+    z = logits(hidden_bits, lm_head_bits) * np.asarray(row_scale, dtype=np.float64)[:, None]
+    mx = z.max(axis=1)
+    lse = mx + np.log(np.exp(z - mx[:, None]).sum(axis=1))
+    return z[np.arange(z.shape[0]), ids] - lse
