@@ -47,6 +47,7 @@ typedef enum {
 /* Bits of the device status word returned by atts_last_device_status. */
 #define ATTS_DEV_TOKEN_ID_RANGE 1u /* a token id was outside [0, V): that row's log-prob is NaN */
 #define ATTS_DEV_WAIT_EXPIRED 2u   /* a pipeline wait in the scoring kernel ran out; outputs invalid */
+#define ATTS_DEV_GROUP_ID_RANGE 4u /* a group id was outside [0, G): that candidate has numer 0 */
 
 /* Stage labels written by atts_classify (the three stages of the rejection-sampling pipeline,
  * Sec. 3.3): the highest stage a sample reaches in this turn. */
@@ -97,6 +98,29 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
                        void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Scoring with a per-row factor on the logits: z_i = row_scale[i] * (W h_i).  This is the LM head applied to
+ * an RMS-normalised hidden state (the step just before the path, Sec. 3.3 "Verification": the target's final
+ * norm) without materialising the normalised copy: row_scale[i] = 1 / sqrt(mean(h_i^2) + eps) from
+ * atts_rms_inv, and the norm's gain vector folded into the columns of lm_head by the caller.  The factor is
+ * folded into the exponent's scale in the epilogue, so the cost is that of atts_score_logprob.
+ *   row_scale     dev  [M] fp32, each finite and > 0 (a row with another value has an undefined result)
+ * Everything else as atts_score_logprob.
+ */
+int atts_score_logprob_scaled(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
+                              const float* row_scale, const int32_t* seg_offsets, int64_t M, int64_t d,
+                              int64_t V, int64_t S, int32_t score_mode, float* token_logprob,
+                              float* sample_score, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream);
+
+/*
+ * row_scale[i] = 1 / sqrt(mean_k hidden[i, k]^2 + eps), fp32 accumulation.
+ *   hidden_bf16   dev  [M, d] bf16 row-major, 16-byte aligned, d a multiple of 8;  eps >= 0
+ *   row_scale     dev  [M] fp32 out
+ */
+int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float* row_scale,
+                 void* cuda_stream);
+
+/*
  * Marginal conformal p-value by rank (Eq. p-value, Proposition 1):
  *   numer[j]  = 1 + #{ i < n : calib_sorted[i] >= scores[j] },  pvalue[j] = numer[j] / (n + 1).
  * Ties count.  A NaN calibration score (sorted last) counts for every candidate; a NaN candidate
@@ -143,6 +167,46 @@ int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, ui
 int atts_rank_classify(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
                        const double* alphas, int32_t n_alpha, uint32_t* numer, float* pvalue,
                        uint8_t* stage, uint32_t* stage_counts, void* cuda_stream);
+
+/*
+ * Threshold form of the acceptance rule (the quantile-threshold construction of the classic set-up,
+ * Eqs. quantile / pred_set, read for the rejection side): with tau = the k_alpha-th largest calibration
+ * score, k_alpha = floor(alpha * (n + 1)), a sample is rejected iff s > tau - exactly the samples with
+ * numer <= k_alpha, ties included.  k_alpha = 0 gives tau = +inf (nobody can be rejected).
+ *   tau           dev  [1] fp32 out
+ */
+int atts_threshold(const float* calib_sorted, int64_t n, double alpha, float* tau, void* cuda_stream);
+
+/*
+ * Stages from one comparison per sample against *tau (no rank, no p-value): ATTS_STAGE_TARGET if s > tau,
+ * ATTS_STAGE_DRAFT if s is NaN, else ATTS_STAGE_ACCEPTED.  Same bytes as atts_conformal_rank followed by
+ * atts_classify for the alpha that produced tau.
+ *   scores dev [Nc] fp32 (16-byte aligned); tau dev [1]; stage dev [Nc] uint8 out (16-byte aligned);
+ *   stage_counts dev [3] uint32 out, overwritten, may be NULL (the third is the budget B)
+ */
+int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, uint8_t* stage,
+                            uint32_t* stage_counts, void* cuda_stream);
+
+/*
+ * Conditional conformal p-value (Proposition 2; Sec. 3.2: "adjusting the comparison with the ... calibration
+ * set from the current input sample"): candidate j is ranked only against the calibration scores of its own
+ * input group_ids[j].  Reading adopted: the same count as the marginal form over the group's scores,
+ *   numer[j] = 1 + #{ i in group : calib[i] >= scores[j] },  denom[j] = |group| + 1,  p = numer / denom.
+ *   scores        dev  [Nc] fp32;  group_ids dev [Nc] int32 in [0, G) (outside: ATTS_DEV_GROUP_ID_RANGE, numer 0)
+ *   calib_segments dev fp32: the groups' scores one after the other, each group ascending (NaNs last)
+ *   seg_offsets   dev  [G + 1] int32, group g is calib_segments[seg_offsets[g] .. seg_offsets[g+1])
+ *   numer, denom  dev  [Nc] uint32 out;  pvalue dev [Nc] fp32 out, may be NULL
+ */
+int atts_conformal_rank_conditional(const float* scores, const int32_t* group_ids, int64_t Nc,
+                                    const float* calib_segments, const int32_t* seg_offsets, int64_t G,
+                                    uint32_t* numer, uint32_t* denom, float* pvalue, void* cuda_stream);
+
+/*
+ * atts_classify with every candidate's own denominator: reject iff 1 <= numer <= floor(alpha * denom)
+ * (IEEE double).  stage / stage_counts as atts_classify.
+ */
+int atts_classify_conditional(const uint32_t* numer, const uint32_t* denom, int64_t Nc, double alpha,
+                              uint8_t* stage, uint32_t* stage_counts, void* cuda_stream);
 
 /* Bytes of workspace atts_calib_update needs to insert k scores into a buffer holding n. */
 int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes);

@@ -17,11 +17,12 @@ EXPORTS = (
     "atts_strerror", "atts_version", "atts_score_workspace_bytes", "atts_score_logprob",
     "atts_conformal_rank", "atts_classify", "atts_calib_workspace_bytes", "atts_calib_update",
     "atts_last_device_status", "atts_profile_begin", "atts_profile_end",
-    "atts_calib_update_static", "atts_rank_classify",
+    "atts_calib_update_static", "atts_rank_classify", "atts_score_logprob_scaled", "atts_rms_inv",
+    "atts_threshold", "atts_classify_threshold", "atts_conformal_rank_conditional", "atts_classify_conditional",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
-DEV_TOKEN_ID_RANGE, DEV_WAIT_EXPIRED = 1, 2
+DEV_TOKEN_ID_RANGE, DEV_WAIT_EXPIRED, DEV_GROUP_ID_RANGE = 1, 2, 4
 
 _lib = None
 
@@ -57,6 +58,14 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.atts_classify.argtypes = [c_void_p, c_int64, c_int64, c_double, c_void_p, c_void_p, c_void_p]
     lib.atts_rank_classify.argtypes = [c_void_p, c_int64, c_void_p, c_int64, POINTER(c_double), c_int32, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_void_p]
+    lib.atts_score_logprob_scaled.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64,
+                                              c_int64, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.atts_rms_inv.argtypes = [c_void_p, c_int64, c_int64, ctypes.c_float, c_void_p, c_void_p]
+    lib.atts_threshold.argtypes = [c_void_p, c_int64, c_double, c_void_p, c_void_p]
+    lib.atts_classify_threshold.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.atts_conformal_rank_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_void_p,
+                                                    c_void_p, c_void_p, c_void_p]
+    lib.atts_classify_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_double, c_void_p, c_void_p, c_void_p]
     lib.atts_calib_workspace_bytes.argtypes = [c_int64, c_int64, POINTER(c_size_t)]
     lib.atts_calib_update.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
                                       c_size_t, c_void_p]
@@ -108,6 +117,48 @@ def score_logprob(hidden, lm_head, token_ids, seg_offsets, token_logprob, sample
     _check(load().atts_score_logprob(_ptr(hidden), _ptr(lm_head), _ptr(token_ids), _ptr(seg_offsets), M, d, V, S,
                                      score_mode, _ptr(token_logprob), _ptr(sample_score), _ptr(workspace),
                                      workspace.numel() * workspace.element_size(), _stream()), "atts_score_logprob")
+
+
+def score_logprob_scaled(hidden, lm_head, token_ids, row_scale, seg_offsets, token_logprob, sample_score, workspace,
+                         score_mode: int = 0) -> None:
+    """score_logprob with logits of row i multiplied by row_scale[i] (f32 [M], finite and > 0)."""
+    M, d = hidden.shape
+    V = lm_head.shape[0]
+    S = seg_offsets.numel() - 1
+    _check(load().atts_score_logprob_scaled(_ptr(hidden), _ptr(lm_head), _ptr(token_ids), _ptr(row_scale),
+                                            _ptr(seg_offsets), M, d, V, S, score_mode, _ptr(token_logprob),
+                                            _ptr(sample_score), _ptr(workspace),
+                                            workspace.numel() * workspace.element_size(), _stream()),
+           "atts_score_logprob_scaled")
+
+
+def rms_inv(hidden, eps: float, row_scale) -> None:
+    """row_scale[i] = 1 / sqrt(mean(hidden[i]^2) + eps)."""
+    M, d = hidden.shape
+    _check(load().atts_rms_inv(_ptr(hidden), M, d, float(eps), _ptr(row_scale), _stream()), "atts_rms_inv")
+
+
+def threshold(calib_sorted, n: int, alpha: float, tau) -> None:
+    """tau[0] = the floor(alpha (n + 1))-th largest of the first n calibration scores (+inf if that is 0)."""
+    _check(load().atts_threshold(_ptr(calib_sorted), n, float(alpha), _ptr(tau), _stream()), "atts_threshold")
+
+
+def classify_threshold(scores, tau, stage, stage_counts=None) -> None:
+    """Stage per sample from s > tau[0]; stage_counts [3] or None."""
+    _check(load().atts_classify_threshold(_ptr(scores), scores.numel(), _ptr(tau), _ptr(stage), _ptr(stage_counts),
+                                          _stream()), "atts_classify_threshold")
+
+
+def conformal_rank_conditional(scores, group_ids, calib_segments, seg_offsets, numer, denom, pvalue=None) -> None:
+    """Rank each score against the ascending calibration segment of its own group."""
+    _check(load().atts_conformal_rank_conditional(_ptr(scores), _ptr(group_ids), scores.numel(), _ptr(calib_segments),
+                                                  _ptr(seg_offsets), seg_offsets.numel() - 1, _ptr(numer), _ptr(denom),
+                                                  _ptr(pvalue), _stream()), "atts_conformal_rank_conditional")
+
+
+def classify_conditional(numer, denom, alpha: float, stage, stage_counts=None) -> None:
+    _check(load().atts_classify_conditional(_ptr(numer), _ptr(denom), numer.numel(), float(alpha), _ptr(stage),
+                                            _ptr(stage_counts), _stream()), "atts_classify_conditional")
 
 
 def conformal_rank(scores, calib_sorted, n: int, numer, pvalue=None) -> None:

@@ -219,10 +219,10 @@ int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_
   return ATTS_OK;
 }
 
-int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
-                       const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V, int64_t S, int32_t score_mode,
-                       float* token_logprob, float* sample_score, void* workspace, size_t workspace_bytes,
-                       void* cuda_stream) {
+static int score_impl(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
+                      const float* row_scale, const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V, int64_t S,
+                      int32_t score_mode, float* token_logprob, float* sample_score, void* workspace,
+                      size_t workspace_bytes, void* cuda_stream) {
   int st = check_score_shape(M, d, V, S);
   if (st != ATTS_OK) return st;
   if (score_mode < 0 || score_mode > 3) return ATTS_ERR_ARG;
@@ -230,7 +230,8 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
   if (M > 0 && (!hidden_bf16 || !token_ids)) return ATTS_ERR_NULL;
   if (S > 0 && !sample_score) return ATTS_ERR_NULL;
   if (!aligned(hidden_bf16, 16) || !aligned(lm_head_bf16, 16) || !aligned(workspace, 256) ||
-      !aligned(token_ids, 4) || !aligned(seg_offsets, 4) || !aligned(token_logprob, 4) || !aligned(sample_score, 4))
+      !aligned(token_ids, 4) || !aligned(seg_offsets, 4) || !aligned(token_logprob, 4) || !aligned(sample_score, 4) ||
+      !aligned(row_scale, 4))
     return ATTS_ERR_ALIGN;
   const DeviceInfo* di;
   st = device_info(&di);
@@ -252,7 +253,7 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
     if (timed) cudaEventRecord(g_prof.ev[2 * g_prof.used], stream);
     if (plan.ctas == 1) {
       const int grid = plan.units < di->sm_count ? plan.units : di->sm_count;
-      lmhead_lse_kernel<1><<<grid, kScoreThreads, ScoreCfg<1>::kSmemBytes, stream>>>(map_h, map_w, token_ids, plan, partial,
+      lmhead_lse_kernel<1><<<grid, kScoreThreads, ScoreCfg<1>::kSmemBytes, stream>>>(map_h, map_w, token_ids, row_scale, plan, partial,
                                                                                      gathered, di->dev_status);
     } else {
       const int pairs = plan.units < di->pair_workers ? plan.units : di->pair_workers;
@@ -268,7 +269,7 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
       attr[0].val.clusterDim.z = 1;
       cfg.attrs = attr;
       cfg.numAttrs = 1;
-      if (cudaLaunchKernelEx(&cfg, lmhead_lse_kernel<2>, map_h, map_w, token_ids, plan, partial, gathered,
+      if (cudaLaunchKernelEx(&cfg, lmhead_lse_kernel<2>, map_h, map_w, token_ids, row_scale, plan, partial, gathered,
                              di->dev_status) != cudaSuccess) {
         cudaGetLastError();
         return ATTS_ERR_CUDA;
@@ -286,6 +287,37 @@ int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const 
     if ((st = launch_status()) != ATTS_OK) return st;
   }
   return ATTS_OK;
+}
+
+int atts_score_logprob(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
+                       const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V, int64_t S, int32_t score_mode,
+                       float* token_logprob, float* sample_score, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream) {
+  return score_impl(hidden_bf16, lm_head_bf16, token_ids, nullptr, seg_offsets, M, d, V, S, score_mode, token_logprob,
+                    sample_score, workspace, workspace_bytes, cuda_stream);
+}
+
+int atts_score_logprob_scaled(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
+                              const float* row_scale, const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V,
+                              int64_t S, int32_t score_mode, float* token_logprob, float* sample_score, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream) {
+  if (M > 0 && !row_scale) return ATTS_ERR_NULL;
+  return score_impl(hidden_bf16, lm_head_bf16, token_ids, row_scale, seg_offsets, M, d, V, S, score_mode, token_logprob,
+                    sample_score, workspace, workspace_bytes, cuda_stream);
+}
+
+int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float* row_scale, void* cuda_stream) {
+  if (M < 0 || M >= (1ll << 31) - kBlockM || d < 8 || d > 65536 || d % 8 != 0) return ATTS_ERR_SHAPE;
+  if (!(eps >= 0.f)) return ATTS_ERR_ARG;
+  if (M > 0 && (!hidden_bf16 || !row_scale)) return ATTS_ERR_NULL;
+  if (!aligned(hidden_bf16, 16) || !aligned(row_scale, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  if (M == 0) return ATTS_OK;
+  rms_inv_kernel<<<(unsigned)((M + 7) / 8), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const uint4*>(hidden_bf16), (int)M, (int)d, eps, row_scale);
+  return launch_status();
 }
 
 // Shared launcher of the rank kernel, with or without the fused thresholding.
@@ -382,6 +414,81 @@ int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, ui
   const int64_t max_blocks = (int64_t)di->sm_count * 8;
   if (blocks > max_blocks) blocks = max_blocks;
   classify_kernel<<<(unsigned)blocks, kClassifyThreads, 0, stream>>>(numer, Nc, k_alpha, stage, stage_counts);
+  return launch_status();
+}
+
+int atts_threshold(const float* calib_sorted, int64_t n, double alpha, float* tau, void* cuda_stream) {
+  if (n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
+  if (!(alpha > 0.0 && alpha < 1.0)) return ATTS_ERR_ARG;
+  if (!tau || (n > 0 && !calib_sorted)) return ATTS_ERR_NULL;
+  if (!aligned(calib_sorted, 4) || !aligned(tau, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  const int k_alpha = (int)floor(alpha * (double)(n + 1));
+  threshold_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(calib_sorted, (int)n, k_alpha, tau);
+  return launch_status();
+}
+
+int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, uint8_t* stage, uint32_t* stage_counts,
+                            void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  if (!tau || (Nc > 0 && (!scores || !stage))) return ATTS_ERR_NULL;
+  if (!aligned(scores, 16) || !aligned(stage, 16) || !aligned(stage_counts, 4) || !aligned(tau, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (stage_counts && cudaMemsetAsync(stage_counts, 0, 3 * sizeof(uint32_t), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  if (Nc == 0) return ATTS_OK;
+  const int64_t per_block = (int64_t)kClassifyThreads * kClassifyPerThread;
+  int64_t blocks = (Nc + per_block - 1) / per_block;
+  const int64_t max_blocks = (int64_t)di->sm_count * 8;
+  if (blocks > max_blocks) blocks = max_blocks;
+  classify_threshold_kernel<<<(unsigned)blocks, kClassifyThreads, 0, stream>>>(scores, Nc, tau, stage, stage_counts);
+  return launch_status();
+}
+
+int atts_conformal_rank_conditional(const float* scores, const int32_t* group_ids, int64_t Nc, const float* calib_segments,
+                                    const int32_t* seg_offsets, int64_t G, uint32_t* numer, uint32_t* denom, float* pvalue,
+                                    void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || G < 0 || G >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  if (Nc > 0 && (!scores || !group_ids || !numer || !denom || !seg_offsets)) return ATTS_ERR_NULL;
+  if (!aligned(scores, 4) || !aligned(group_ids, 4) || !aligned(numer, 4) || !aligned(denom, 4) || !aligned(pvalue, 4) ||
+      !aligned(calib_segments, 4) || !aligned(seg_offsets, 4))
+    return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  if (Nc == 0) return ATTS_OK;
+  int64_t blocks = (Nc + 255) / 256;
+  if (blocks > (int64_t)di->sm_count * 8) blocks = (int64_t)di->sm_count * 8;
+  rank_conditional_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      scores, group_ids, Nc, calib_segments, seg_offsets, (int)G, numer, denom, pvalue, di->dev_status);
+  return launch_status();
+}
+
+int atts_classify_conditional(const uint32_t* numer, const uint32_t* denom, int64_t Nc, double alpha, uint8_t* stage,
+                              uint32_t* stage_counts, void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  if (!(alpha > 0.0 && alpha < 1.0)) return ATTS_ERR_ARG;
+  if (Nc > 0 && (!numer || !denom || !stage)) return ATTS_ERR_NULL;
+  if (!aligned(numer, 4) || !aligned(denom, 4) || !aligned(stage_counts, 4)) return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (stage_counts && cudaMemsetAsync(stage_counts, 0, 3 * sizeof(uint32_t), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  if (Nc == 0) return ATTS_OK;
+  int64_t blocks = (Nc + 255) / 256;
+  if (blocks > (int64_t)di->sm_count * 8) blocks = (int64_t)di->sm_count * 8;
+  classify_conditional_kernel<<<(unsigned)blocks, 256, 0, stream>>>(numer, denom, Nc, alpha, stage, stage_counts);
   return launch_status();
 }
 

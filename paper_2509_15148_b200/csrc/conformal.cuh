@@ -366,4 +366,119 @@ merge_kernel(const float* __restrict__ old_buf, int n, const uint32_t* __restric
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Threshold form of the acceptance rule: tau = the k_alpha-th largest calibration score, and a sample is
+// rejected iff s > tau (identical to numer <= k_alpha, ties included).  One comparison per sample.
+// ---------------------------------------------------------------------------------------------
+__global__ void threshold_kernel(const float* __restrict__ calib, int n, int k_alpha, float* __restrict__ tau) {
+  if (threadIdx.x == 0 && blockIdx.x == 0) *tau = k_alpha >= 1 ? calib[n - k_alpha] : __uint_as_float(0x7F800000u);
+}
+
+__global__ void __launch_bounds__(kClassifyThreads)
+classify_threshold_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restrict__ tau_ptr,
+                          uint8_t* __restrict__ stage, uint32_t* __restrict__ counts) {
+  const float tau = __ldg(tau_ptr);
+  uint32_t c1 = 0, c3 = 0, cnt = 0;
+  auto st_of = [&](float s) { return s != s ? 1u : (s > tau ? 3u : 2u); };
+  const int64_t per_block = (int64_t)kClassifyThreads * kClassifyPerThread;
+  for (int64_t base = (int64_t)blockIdx.x * per_block; base < Nc; base += (int64_t)gridDim.x * per_block) {
+    const int64_t j = base + (int64_t)threadIdx.x * kClassifyPerThread;
+    if (j + kClassifyPerThread <= Nc) {
+      uint32_t packed[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(scores + j + 4 * q);
+        const uint32_t s0 = st_of(v.x), s1 = st_of(v.y), s2 = st_of(v.z), s3 = st_of(v.w);
+        c1 += (s0 == 1u) + (s1 == 1u) + (s2 == 1u) + (s3 == 1u);
+        c3 += (s0 == 3u) + (s1 == 3u) + (s2 == 3u) + (s3 == 3u);
+        packed[q] = s0 | (s1 << 8) | (s2 << 16) | (s3 << 24);
+      }
+      cnt += kClassifyPerThread;
+      *reinterpret_cast<uint4*>(stage + j) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    } else {
+      for (int e = 0; e < kClassifyPerThread && j + e < Nc; ++e) {
+        const uint32_t s = st_of(scores[j + e]);
+        c1 += (s == 1u);
+        c3 += (s == 3u);
+        cnt += 1;
+        stage[j + e] = (uint8_t)s;
+      }
+    }
+  }
+  if (counts == nullptr) return;
+  uint32_t c2 = cnt - c1 - c3;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    c1 += __shfl_xor_sync(0xFFFFFFFFu, c1, o);
+    c2 += __shfl_xor_sync(0xFFFFFFFFu, c2, o);
+    c3 += __shfl_xor_sync(0xFFFFFFFFu, c3, o);
+  }
+  __shared__ uint32_t sh[3][kClassifyThreads / 32];
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  if (l == 0) { sh[0][w] = c1; sh[1][w] = c2; sh[2][w] = c3; }
+  __syncthreads();
+  if (threadIdx.x < 3) {
+    uint32_t t = 0;
+    for (int i = 0; i < kClassifyThreads / 32; ++i) t += sh[threadIdx.x][i];
+    if (t) atomicAdd(counts + threadIdx.x, t);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Conditional coverage (Proposition 2): a candidate is ranked against the calibration scores of its own
+// input only.  The per-input buffers are ascending segments of one array; segments are short (the m samples
+// of one input), so a thread searches its segment directly in (L2-resident) global memory.
+//   numer = 1 + #{own segment >= s},  denom = |segment| + 1,  p = numer / denom;  reject iff
+//   1 <= numer <= floor(alpha * denom)  (evaluated in IEEE double, as on the host for the marginal form).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restrict__ group_ids, int64_t Nc,
+                        const float* __restrict__ calib, const int32_t* __restrict__ seg_offsets, int G,
+                        uint32_t* __restrict__ numer, uint32_t* __restrict__ denom, float* __restrict__ pvalue,
+                        unsigned int* __restrict__ dev_status) {
+  for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < Nc; j += (int64_t)gridDim.x * 256) {
+    const float s = scores[j];
+    const int g = group_ids[j];
+    uint32_t num = 0u, den = 1u;
+    if (g < 0 || g >= G) {
+      atomicOr(dev_status, 4u);  // group id out of range: no calibration set, treated as "no score"
+    } else {
+      const int a = __ldg(seg_offsets + g), b = __ldg(seg_offsets + g + 1);
+      den = (uint32_t)(b - a) + 1u;
+      if (s == s) {
+        int lo = a, len = b - a;  // first entry of the segment that is not below s
+        while (len > 0) {
+          const int half = len >> 1;
+          const bool less = __ldg(calib + lo + half) < s;
+          lo = less ? lo + half + 1 : lo;
+          len = less ? len - half - 1 : half;
+        }
+        num = (uint32_t)(b - lo) + 1u;
+      }
+    }
+    numer[j] = num;
+    denom[j] = den;
+    if (pvalue) pvalue[j] = num ? __fdiv_rn((float)num, (float)den) : __uint_as_float(0x7FC00000u);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+classify_conditional_kernel(const uint32_t* __restrict__ numer, const uint32_t* __restrict__ denom, int64_t Nc,
+                            double alpha, uint8_t* __restrict__ stage, uint32_t* __restrict__ counts) {
+  uint32_t c[3] = {0, 0, 0};
+  for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < Nc; j += (int64_t)gridDim.x * 256) {
+    const uint32_t k_alpha = (uint32_t)floor(alpha * (double)denom[j]);
+    const uint32_t s = stage_of(numer[j], k_alpha);
+    stage[j] = (uint8_t)s;
+    c[s - 1] += 1;
+  }
+  if (counts == nullptr) return;
+#pragma unroll
+  for (int i = 0; i < 3; ++i) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c[i] += __shfl_xor_sync(0xFFFFFFFFu, c[i], o);
+    if ((threadIdx.x & 31) == 0 && c[i]) atomicAdd(counts + i, c[i]);
+  }
+}
+
 }  // namespace atts

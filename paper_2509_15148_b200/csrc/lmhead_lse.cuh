@@ -254,7 +254,7 @@ __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.
 template <int CTAS>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
-                  const int32_t* __restrict__ token_ids, const ScorePlan plan,
+                  const int32_t* __restrict__ token_ids, const float* __restrict__ row_scale, const ScorePlan plan,
                   float2* __restrict__ partial, float* __restrict__ gathered, unsigned int* __restrict__ dev_status) {
   using Cfg = ScoreCfg<CTAS>;
   constexpr int kStages = Cfg::kStages;
@@ -390,6 +390,10 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
       decode_unit(plan, u, rb, c, nt0, nt1);
       const int row = rb * Cfg::kRowsPerUnit + (int)rank * kBlockM + quarter * 32 + lane;
       const int y = (row < plan.M) ? token_ids[row] : -1;
+      // optional per-row factor on the logits (finite, > 0): folded into the exponent's scale, so it costs nothing per
+      // element; the running maximum is kept on the unscaled logits
+      const float rs = (row_scale != nullptr && row < plan.M) ? row_scale[row] : 1.f;
+      const float kScale = rs * kLog2e;
       float m = -INFINITY, l = 0.f;
       for (int nt = nt0; nt < nt1; ++nt) {
         if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
@@ -414,20 +418,20 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
 #pragma unroll
             for (int i = 0; i < 32; ++i)
               if (i == yi) g = __uint_as_float(v[i]);
-            gathered[row] = g;
+            gathered[row] = g * rs;
           }
           float cmax = __uint_as_float(v[0]);
 #pragma unroll
           for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, __uint_as_float(v[i]));
           const float m_new = fmaxf(m, cmax);
-          const float ms = m_new * kLog2e;
+          const float ms = m_new * kScale;
           float s0 = 0.f, s1 = 0.f;
 #pragma unroll
           for (int i = 0; i < 32; i += 2) {
-            s0 += ex2_approx(fmaf(__uint_as_float(v[i]), kLog2e, -ms));
-            s1 += ex2_approx(fmaf(__uint_as_float(v[i + 1]), kLog2e, -ms));
+            s0 += ex2_approx(fmaf(__uint_as_float(v[i]), kScale, -ms));
+            s1 += ex2_approx(fmaf(__uint_as_float(v[i + 1]), kScale, -ms));
           }
-          l = l * ex2_approx((m - m_new) * kLog2e) + (s0 + s1);
+          l = l * ex2_approx((m - m_new) * kScale) + (s0 + s1);
           m = m_new;
         }
         tc_fence_before();
@@ -439,7 +443,7 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
         acc ^= 1;
         if (acc == 0) acc_phase ^= 1u;
       }
-      if (ok && row < plan.M) partial[(size_t)c * plan.M_pad + row] = make_float2(m, l);
+      if (ok && row < plan.M) partial[(size_t)c * plan.M_pad + row] = make_float2(m * rs, l);
     }
   }
 
@@ -458,6 +462,33 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
     if (CTAS == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
     else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTmemCols) : "memory");
   }
+}
+
+// ------------------------------------------------------------------------------------------
+// Row factor of an RMS normalisation: out[i] = 1 / sqrt(mean_k h[i, k]^2 + eps).  One warp per row, 128-bit
+// loads, fp32 accumulation in a fixed order.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+rms_inv_kernel(const uint4* __restrict__ hidden, int M, int d, float eps, float* __restrict__ out) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (row >= M) return;
+  const int lane = threadIdx.x & 31;
+  const int vecs = d / 8;  // 8 bf16 per 16 bytes
+  const uint4* p = hidden + (size_t)row * vecs;
+  float acc = 0.f;
+  for (int i = lane; i < vecs; i += 32) {
+    const uint4 q = __ldg(p + i);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float lo = __uint_as_float(w[t] << 16), hi = __uint_as_float(w[t] & 0xFFFF0000u);
+      acc = fmaf(lo, lo, acc);
+      acc = fmaf(hi, hi, acc);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  if (lane == 0) out[row] = rsqrtf(acc / (float)d + eps);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -1,0 +1,110 @@
+"""GPU parity of the extension entry points (threshold form, conditional coverage, row-scaled scoring)
+against the CPU oracle, through the C-ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import atts_oracle as orc
+from paper_2509_15148_b200 import binding, inputs
+from tests.gpu_util import dev, dev_bf16, f32_bits, host_u32, poison, workspace
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("alpha", [0.01, 0.1, 0.25, 0.9])
+@pytest.mark.parametrize("Nc,n", [(5, 8), (4099, 400), (300000, 65536)])
+def test_threshold_classify_equals_rank_classify(alpha, Nc, n):
+    calib = np.sort(np.round(inputs.lognormal_scores(10 + n, n), 2))             # ties
+    scores = np.round(inputs.lognormal_scores(20 + Nc, Nc), 2)
+    scores[: min(Nc, 4)] = np.array([np.nan, np.inf, -np.inf, calib[-1]], np.float32)[: min(Nc, 4)]
+    c_dev, s_dev = dev(calib), dev(scores)
+    tau = poison((1,), torch.float32)
+    binding.threshold(c_dev, n, alpha, tau)
+    stage = poison((Nc,), torch.uint8)
+    counts = poison((3,), torch.int32)
+    binding.classify_threshold(s_dev, tau, stage, counts)
+    torch.cuda.synchronize()
+    want_tau = orc.threshold(calib, alpha)
+    assert f32_bits(tau)[0] == f32_bits(np.array([want_tau], np.float32))[0]
+    want_stage, want_counts = orc.classify_by_threshold(scores, want_tau)
+    assert np.array_equal(stage.cpu().numpy(), want_stage)
+    assert np.array_equal(host_u32(counts), want_counts)
+    # the same bytes as the rank route
+    numer = poison((Nc,), torch.int32)
+    stage2 = poison((Nc,), torch.uint8)
+    binding.conformal_rank(s_dev, c_dev, n, numer, None)
+    binding.classify(numer, n, alpha, stage2, None)
+    torch.cuda.synchronize()
+    assert torch.equal(stage, stage2)
+
+
+def test_conditional_rank_and_classify_bit_exact():
+    rng = np.random.default_rng(3)
+    G = 300
+    sizes = rng.integers(0, 130, size=G)
+    sizes[:3] = [0, 1, 128]
+    groups = [np.sort(np.round(inputs.lognormal_scores(100 + g, int(sizes[g])), 1)) for g in range(G)]
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    calib = np.concatenate(groups).astype(np.float32)
+    Nc = 20000
+    gid = rng.integers(0, G, size=Nc).astype(np.int32)
+    gid[:3] = [0, 1, 2]
+    scores = np.round(inputs.lognormal_scores(7, Nc), 1)
+    scores[5] = np.nan
+    numer = poison((Nc,), torch.int32)
+    denom = poison((Nc,), torch.int32)
+    p = poison((Nc,), torch.float32)
+    binding.conformal_rank_conditional(dev(scores), dev(gid), dev(calib), dev(off), numer, denom, p)
+    want_numer, want_denom = orc.conformal_numer_conditional(scores, gid, groups)
+    assert np.array_equal(host_u32(numer), want_numer)
+    assert np.array_equal(host_u32(denom), want_denom)
+    want_p = (want_numer.astype(np.float64) / want_denom.astype(np.float64)).astype(np.float32)
+    want_p[want_numer == 0] = np.nan
+    assert np.array_equal(f32_bits(p), f32_bits(want_p))
+    for alpha in (0.1, 0.25, 0.5):
+        stage = poison((Nc,), torch.uint8)
+        counts = poison((3,), torch.int32)
+        binding.classify_conditional(numer, denom, alpha, stage, counts)
+        want_stage, want_counts = orc.classify_conditional(want_numer, want_denom, alpha)
+        assert np.array_equal(stage.cpu().numpy(), want_stage)
+        assert np.array_equal(host_u32(counts), want_counts)
+    assert binding.last_device_status() == 0
+    # a group id out of range is flagged, not fatal
+    gid2 = gid.copy()
+    gid2[10] = G
+    binding.conformal_rank_conditional(dev(scores), dev(gid2), dev(calib), dev(off), numer, denom, None)
+    assert binding.last_device_status() & binding.DEV_GROUP_ID_RANGE
+    assert host_u32(numer)[10] == 0
+
+
+@pytest.mark.parametrize("M,d,V", [(300, 192, 1000), (1000, 512, 5000), (4096, 1024, 8192)])
+def test_rms_inv_and_scaled_scoring(M, d, V):
+    rng = np.random.default_rng(M)
+    raw = rng.standard_normal((M, d)).astype(np.float32) * rng.uniform(0.2, 6.0, size=(M, 1)).astype(np.float32)
+    Hb = inputs.f32_to_bf16_bits(raw)                                   # un-normalised hidden states
+    Wb = inputs.lm_head(2, V, d)
+    ids = inputs.zipf_ids(3, M, V)
+    off = np.array([0, M // 2, M], np.int32)
+    H = dev_bf16(Hb)
+    rs = poison((M,), torch.float32)
+    binding.rms_inv(H, 1e-6, rs)
+    torch.cuda.synchronize()
+    want_rs = orc.rms_inv(Hb, 1e-6)
+    assert np.abs(rs.cpu().numpy() / want_rs - 1).max() < 1e-5
+    lp = poison((M,), torch.float32)
+    sc = poison((2,), torch.float32)
+    ws = workspace(binding.score_workspace_bytes(M, d, V, 2))
+    binding.score_logprob_scaled(H, dev_bf16(Wb), dev(ids), rs, dev(off), lp, sc, ws)
+    assert binding.last_device_status() == 0
+    # the oracle gets the device's fp32 row factors, so that only the scoring arithmetic is compared
+    want = orc.token_logprob_scaled(Hb, Wb, ids, rs.cpu().numpy().astype(np.float64))
+    assert np.abs(lp.cpu().numpy() - want).max() <= 2e-3
+    assert np.abs(sc.cpu().numpy() - orc.sample_score(want, off)).max() <= 2e-3
+    # scale 1 reproduces the unscaled entry point bit for bit
+    ones = torch.ones(M, device="cuda")
+    lp1 = poison((M,), torch.float32)
+    lp2 = poison((M,), torch.float32)
+    binding.score_logprob_scaled(H, dev_bf16(Wb), dev(ids), ones, dev(off), lp1, sc, ws)
+    binding.score_logprob(H, dev_bf16(Wb), dev(ids), dev(off), lp2, sc, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(lp1, lp2)
