@@ -189,27 +189,7 @@ def conformal_stress(torch, binding, peaks):
             n = binding.calib_update(buf, n, news[t], ws)
         return n
 
-    def graph_ms(fn, reps=1, rounds=5):
-        """GPU time of fn(): captured `reps` times into one CUDA graph, best of `rounds` replays (events around the
-        replay), so that host launch overhead between these microsecond kernels is not what is measured."""
-        fn()
-        torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g):
-            for _ in range(reps):
-                fn()
-        g.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        best = float("inf")
-        for _ in range(rounds):
-            e0.record()
-            g.replay()
-            e1.record()
-            torch.cuda.synchronize()
-            best = min(best, e0.elapsed_time(e1))
-        return best / reps
-
+    graph_ms = make_graph_timer(torch)
     ms_seq = graph_ms(sequence)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     eager = []
@@ -242,6 +222,41 @@ def conformal_stress(torch, binding, peaks):
         "rank_classify_fused_us": ms_fused * 1e3, "rank_classify_fused_gbs": fused_bytes / (ms_fused * 1e-3) / 1e9,
     }
     del scores, numer, p, stage, stage3
+    out.update(conformal_scaled(torch, binding, peaks, graph_ms))
+    return out
+
+
+def make_graph_timer(torch):
+    def graph_ms(fn, reps=1, rounds=5):
+        """GPU time of fn(): captured `reps` times into one CUDA graph, best of `rounds` replays (events around the
+        replay), so that host launch overhead between these microsecond kernels is not what is measured."""
+        fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(reps):
+                fn()
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        best = float("inf")
+        for _ in range(rounds):
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return best / reps
+    return graph_ms
+
+
+def conformal_scaled(torch, binding, peaks, graph_ms):
+    """The conformal kernels at sizes where HBM is the limit (extra points, not a BASELINE config)."""
+    dev = "cuda"
+    out = {}
+    k = inputs.CONFORMAL_STRESS["k"]
+    counts = torch.empty(3, dtype=torch.int32, device=dev)
+    new0 = torch.from_numpy(inputs.lognormal_scores(inputs.BASE_SEED + 3, k)).to(dev)
     # The same kernels where HBM is the limit: 2^26 candidates (805 MB of traffic per rank pass) against the
     # model-sized buffer n = 4096, and a merge-insert into a 2^22-entry buffer.
     big, n_small = 1 << 26, 4096
@@ -278,7 +293,7 @@ def conformal_stress(torch, binding, peaks):
     bufb = torch.empty(n_big + k, device=dev)
     bufb[:n_big] = torch.sort(torch.randn(n_big, device=dev, generator=gen).exp_()).values
     wsb = torch.empty(binding.calib_workspace_bytes(n_big, k), dtype=torch.uint8, device=dev)
-    ms = graph_ms(lambda: binding.calib_update(bufb, n_big, news[0], wsb), reps=2)
+    ms = graph_ms(lambda: binding.calib_update(bufb, n_big, new0, wsb), reps=2)
     upd_bytes = 16.0 * (n_big + k)   # merge: read + write; copy back: read + write
     out["scaled_update"] = {"n": n_big, "k": k, "us": ms * 1e3, "gbs": upd_bytes / (ms * 1e-3) / 1e9,
                             "frac_hbm": upd_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -302,9 +317,11 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     binding.load()
     peaks, peak_kind = measured_peaks()
-    if args.conformal_only:
+    if args.conformal_only or args.conformal_scaled_only:
         if rank == 0:
-            print(json.dumps({"conformal_stress": conformal_stress(torch, binding, peaks)}), flush=True)
+            res = (conformal_scaled(torch, binding, peaks, make_graph_timer(torch)) if args.conformal_scaled_only
+                   else conformal_stress(torch, binding, peaks))
+            print(json.dumps({"conformal_stress": res}), flush=True)
         return
 
     c = inputs.CONFIGS[args.workload]
@@ -517,6 +534,8 @@ def main():
                     help="shape to run (default: the bench line's workload; others are for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-conformal", action="store_true")
+    ap.add_argument("--conformal-scaled-only", action="store_true",
+                    help="run only the HBM-scale points of the conformal kernels (for profiling)")
     ap.add_argument("--conformal-only", action="store_true",
                     help="run only the conformal-only workload section and print it (for profiling those kernels)")
     args = ap.parse_args()
