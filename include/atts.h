@@ -83,7 +83,8 @@ int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_
  *                      yields NaN for that row
  *   seg_offsets   dev  [S + 1] int32, 0 = o_0 <= o_1 <= ... <= o_S = M (not checked on the device
  *                      beyond clamping to [0, M])
- *   M, d, V, S         0 <= M < 2^31, d a multiple of 64 with 64 <= d <= 65536, 1 <= V < 2^31,
+ *   M, d, V, S         0 <= M < 2^31, d a multiple of 64 with 64 <= d <= 16384 (the fp32 accumulation error of
+ *                      a logit grows with d; 2e-3 on the log-probs was verified up to this size), 1 <= V < 2^31,
  *                      0 <= S
  *   token_logprob dev  [M] fp32 out, may be NULL
  *   sample_score  dev  [S] fp32 out, may be NULL when S == 0
@@ -267,6 +268,18 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
  * ATTS_ERR_TIMEOUT if ATTS_DEV_WAIT_EXPIRED is among them, else ATTS_OK.
  */
 int atts_last_device_status(void* cuda_stream, uint32_t* bits);
+
+/*
+ * Schedule inspection (diagnostic; the paper has no counterpart; needs no device).  The static schedule the
+ * fused kernel would use for M x d x V with `workers` concurrent workers of `ctas` (1 or 2) CTAs each:
+ *   atts_debug_score_plan: out[0..8) = {row blocks, vocabulary tiles, k blocks, chunks per row block,
+ *                          row blocks per panel, units, padded rows, ctas}
+ *   atts_debug_score_unit: out[0..4) = {row block, chunk, first tile, one past the last tile} of unit u
+ * Both return ATTS_ERR_SHAPE / ATTS_ERR_ARG for sizes atts_score_logprob would reject.
+ */
+int atts_debug_score_plan(int64_t M, int64_t d, int64_t V, int32_t workers, int32_t ctas, int32_t* out);
+int atts_debug_score_unit(int64_t M, int64_t d, int64_t V, int32_t workers, int32_t ctas, int32_t u,
+                          int32_t* out);
 
 /*
  * Timing hooks (measurement aid; the paper has no counterpart).  Between atts_profile_begin and

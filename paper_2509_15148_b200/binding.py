@@ -19,6 +19,7 @@ EXPORTS = (
     "atts_last_device_status", "atts_profile_begin", "atts_profile_end",
     "atts_calib_update_static", "atts_rank_classify", "atts_score_logprob_scaled", "atts_rms_inv",
     "atts_threshold", "atts_classify_threshold", "atts_conformal_rank_conditional", "atts_classify_conditional",
+    "atts_debug_score_plan", "atts_debug_score_unit",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -66,6 +67,8 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.atts_conformal_rank_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_void_p,
                                                     c_void_p, c_void_p, c_void_p]
     lib.atts_classify_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_double, c_void_p, c_void_p, c_void_p]
+    lib.atts_debug_score_plan.argtypes = [c_int64, c_int64, c_int64, c_int32, c_int32, POINTER(c_int32)]
+    lib.atts_debug_score_unit.argtypes = [c_int64, c_int64, c_int64, c_int32, c_int32, c_int32, POINTER(c_int32)]
     lib.atts_calib_workspace_bytes.argtypes = [c_int64, c_int64, POINTER(c_size_t)]
     lib.atts_calib_update.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
                                       c_size_t, c_void_p]
@@ -235,3 +238,17 @@ def profile_end(cap: int = 4096) -> list[float]:
     cnt = c_int(0)
     _check(load().atts_profile_end(buf, cap, ctypes.byref(cnt)), "atts_profile_end")
     return [float(buf[i]) for i in range(min(cnt.value, cap))]
+
+
+def debug_score_plan(M: int, d: int, V: int, workers: int, ctas: int) -> dict:
+    """The fused kernel's static schedule for a shape (no device needed)."""
+    out = (c_int32 * 8)()
+    _check(load().atts_debug_score_plan(M, d, V, workers, ctas, out), "atts_debug_score_plan")
+    return dict(zip(("RB", "NT", "KB", "C", "Gr", "units", "M_pad", "ctas"), list(out)))
+
+
+def debug_score_unit(M: int, d: int, V: int, workers: int, ctas: int, u: int) -> tuple:
+    """(row block, chunk, first tile, one past the last tile) of unit u of that schedule."""
+    out = (c_int32 * 4)()
+    _check(load().atts_debug_score_unit(M, d, V, workers, ctas, u, out), "atts_debug_score_unit")
+    return tuple(out)

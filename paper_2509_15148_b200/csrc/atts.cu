@@ -139,7 +139,7 @@ static ScorePlan choose_score_plan(const DeviceInfo* di, int64_t M, int64_t d, i
 
 static int check_score_shape(int64_t M, int64_t d, int64_t V, int64_t S) {
   if (M < 0 || M >= (1ll << 31) - kBlockM || S < 0 || S >= (1ll << 31)) return ATTS_ERR_SHAPE;
-  if (d < 64 || d > 65536 || d % 64 != 0) return ATTS_ERR_SHAPE;
+  if (d < 64 || d > 16384 || d % 64 != 0) return ATTS_ERR_SHAPE;
   if (V < 1 || V >= (1ll << 31) - kBlockN) return ATTS_ERR_SHAPE;
   return ATTS_OK;
 }
@@ -307,7 +307,7 @@ int atts_score_logprob_scaled(const void* hidden_bf16, const void* lm_head_bf16,
 }
 
 int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float* row_scale, void* cuda_stream) {
-  if (M < 0 || M >= (1ll << 31) - kBlockM || d < 8 || d > 65536 || d % 8 != 0) return ATTS_ERR_SHAPE;
+  if (M < 0 || M >= (1ll << 31) - kBlockM || d < 8 || d > 16384 || d % 8 != 0) return ATTS_ERR_SHAPE;
   if (!(eps >= 0.f)) return ATTS_ERR_ARG;
   if (M > 0 && (!hidden_bf16 || !row_scale)) return ATTS_ERR_NULL;
   if (!aligned(hidden_bf16, 16) || !aligned(row_scale, 4)) return ATTS_ERR_ALIGN;
@@ -591,6 +591,30 @@ int atts_last_device_status(void* cuda_stream, uint32_t* bits) {
   }
   *bits = v;
   return (v & ATTS_DEV_WAIT_EXPIRED) ? ATTS_ERR_TIMEOUT : ATTS_OK;
+}
+
+int atts_debug_score_plan(int64_t M, int64_t d, int64_t V, int32_t workers, int32_t ctas, int32_t* out) {
+  if (!out) return ATTS_ERR_NULL;
+  int st = check_score_shape(M, d, V, 0);
+  if (st != ATTS_OK) return st;
+  if (workers < 1 || (ctas != 1 && ctas != 2)) return ATTS_ERR_ARG;
+  const ScorePlan p = make_score_plan(M, d, V, workers, ctas);
+  const int32_t v[8] = {p.RB, p.NT, p.KB, p.C, p.Gr, p.units, p.M_pad, p.ctas};
+  for (int i = 0; i < 8; ++i) out[i] = v[i];
+  return ATTS_OK;
+}
+
+int atts_debug_score_unit(int64_t M, int64_t d, int64_t V, int32_t workers, int32_t ctas, int32_t u, int32_t* out) {
+  if (!out) return ATTS_ERR_NULL;
+  int st = check_score_shape(M, d, V, 0);
+  if (st != ATTS_OK) return st;
+  if (workers < 1 || (ctas != 1 && ctas != 2)) return ATTS_ERR_ARG;
+  const ScorePlan p = make_score_plan(M, d, V, workers, ctas);
+  if (u < 0 || u >= p.units) return ATTS_ERR_ARG;
+  int rb, c, nt0, nt1;
+  decode_unit(p, u, rb, c, nt0, nt1);
+  out[0] = rb; out[1] = c; out[2] = nt0; out[3] = nt1;
+  return ATTS_OK;
 }
 
 int atts_profile_begin(int max_records) {

@@ -73,6 +73,25 @@ def test_shapes_tiles_and_ragged_tails(M, d, V):
     check_against_oracle(Hb, Wb, ids, off)
 
 
+def test_maximum_hidden_size_long_k_loop():
+    # d = 16384 is the largest hidden size accepted: 256 k-blocks per tile, dozens of ring wraps
+    M, d, V = 130, 16384, 300
+    Hb, Wb = inputs.hidden(41, M, d), inputs.lm_head(42, V, d)
+    ids = inputs.zipf_ids(43, M, V)
+    check_against_oracle(Hb, Wb, ids, np.array([0, 100, M], np.int32))
+
+
+def test_several_l2_panels_single_cta_schedule():
+    # H = 63 MB: more than one L2 panel, so the single-CTA schedule runs with several panels and a ragged last one
+    M, d, V = 15000, 2112, 1300
+    Hb, Wb = inputs.hidden(51, M, d), inputs.lm_head(52, V, d)
+    ids = inputs.zipf_ids(53, M, V)
+    off = inputs.ragged_seg_offsets(54, 40, 700)
+    off = np.minimum(off, M).astype(np.int32)
+    off[-1] = M
+    check_against_oracle(Hb, Wb, ids, off)
+
+
 def test_token_ids_at_tile_edges():
     M, d, V = 256, 128, 1500
     Hb = inputs.hidden(1, M, d)
@@ -152,6 +171,13 @@ def test_run_to_run_bit_identical():
     b = gpu_score(Hb, Wb, ids, off)
     assert np.array_equal(a[0].view(np.uint32), b[0].view(np.uint32))
     assert np.array_equal(a[1].view(np.uint32), b[1].view(np.uint32))
+
+
+def test_hidden_size_beyond_the_limit_is_rejected():
+    import ctypes
+    sz = ctypes.c_size_t(0)
+    assert binding.load().atts_score_workspace_bytes(128, 16384 + 64, 256, 1, ctypes.byref(sz)) == 2
+    assert binding.load().atts_score_workspace_bytes(128, 16384, 256, 1, ctypes.byref(sz)) == 0
 
 
 def test_argument_errors_on_device():
