@@ -34,7 +34,7 @@ ALPHA = 0.1
 METRIC = "draft tokens scored/s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-KERNELS_PER_STEP = 7  # lmhead_lse, lse_combine, segment_score, rank, classify, sort_new, merge
+KERNELS_PER_STEP = 6  # lmhead_lse, lse_combine, segment_score, rank, classify, small_update (n + k small: one block)
 # DRAM bytes per launch of the fused kernel on this workload, from an ncu capture (profiles/), valid only for
 # the kernel source it was taken on: (sha256 of csrc/lmhead_lse.cuh, dram__bytes_read.sum + dram__bytes_write.sum).
 K1_TRAFFIC = ("f0d03bf8bca545c8b7efc61d7700aa660e4822ad071399417aff8f14c1b8fe1b", 8.078e10)
@@ -251,7 +251,7 @@ def make_graph_timer(torch):
 
 
 def conformal_scaled(torch, binding, peaks, graph_ms):
-    """The conformal kernels at sizes where HBM is the limit (extra points, not a BASELINE config)."""
+    """The conformal kernels at sizes where HBM is the limit (extra points beside the five workload shapes)."""
     dev = "cuda"
     out = {}
     k = inputs.CONFORMAL_STRESS["k"]

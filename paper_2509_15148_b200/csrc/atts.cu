@@ -83,6 +83,8 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaFuncSetAttribute(rank_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kSortMaxK * 4) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(small_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      4 * (kSmallUpdMaxOld + kSmallUpdMaxNew)) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kSortMaxK * 4) == cudaSuccess;
       if (!ok) {
@@ -519,6 +521,13 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
   const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
   uint32_t* sorted_keys = static_cast<uint32_t*>(workspace);
   float* merged = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up((size_t)kk * 4, 256));
+  // Small problems: one block does it in place in one launch.
+  if (n <= kSmallUpdMaxOld && k <= kSmallUpdMaxNew && k * 8 <= n + 64) {
+    int k2 = 1;
+    while (k2 < k) k2 <<= 1;
+    small_update_kernel<<<1, kSmallUpdThreads, (size_t)4 * (k2 + n), stream>>>(calib, (int)n, new_scores, (int)k, k2);
+    return launch_status();
+  }
   // Sort the new keys, merge into the workspace, copy back.  Batches larger than one sort launch handles are
   // inserted slice by slice.
   int64_t cur = n;

@@ -481,4 +481,64 @@ classify_conditional_kernel(const uint32_t* __restrict__ numer, const uint32_t* 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// K5+K6 for small problems (the model configurations: a few thousand calibration scores, tens of new ones):
+// one block, one launch, truly in place, no workspace.  The block sorts the new keys in shared memory
+// (bitonic network over k2 = k rounded up to a power of two, padded with a key above every canonical key),
+// copies the old buffer into shared memory, and after a barrier - every read of the old buffer is done -
+// writes each element to its merged slot (old[i] -> i + #{new < old[i]}, new[j] -> j + #{old <= new[j]}).
+// ---------------------------------------------------------------------------------------------
+constexpr int kSmallUpdThreads = 1024;
+constexpr int kSmallUpdMaxOld = 28672;  // 112 KB of shared memory
+constexpr int kSmallUpdMaxNew = 4096;   // 16 KB
+
+__global__ void __launch_bounds__(kSmallUpdThreads, 1)
+small_update_kernel(float* calib, int n, const float* __restrict__ new_scores, int k, int k2) {
+  extern __shared__ uint32_t sm[];
+  uint32_t* nk = sm;        // [k2] sorted new keys
+  uint32_t* ok = sm + k2;   // [n] keys of the old buffer
+  for (int t = threadIdx.x; t < k2; t += kSmallUpdThreads)
+    nk[t] = t < k ? key_of_bits(canonical_bits(new_scores[t])) : 0xFFFFFFFFu;
+  for (int t = threadIdx.x; t < n; t += kSmallUpdThreads) ok[t] = key_of_bits(canonical_bits(calib[t]));
+  __syncthreads();
+  for (int size = 2; size <= k2; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = threadIdx.x; t < (k2 >> 1); t += kSmallUpdThreads) {
+        const int lo = 2 * t - (t & (stride - 1));
+        const int hi = lo + stride;
+        const uint32_t a = nk[lo], b = nk[hi];
+        if ((a > b) == ((lo & size) == 0)) {
+          nk[lo] = b;
+          nk[hi] = a;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  for (int e = threadIdx.x; e < n + k; e += kSmallUpdThreads) {
+    if (e < n) {
+      const uint32_t key = ok[e];
+      int lo = 0, len = k;  // number of new keys < key
+      while (len > 0) {
+        const int half = len >> 1;
+        const bool less = nk[lo + half] < key;
+        lo = less ? lo + half + 1 : lo;
+        len = less ? len - half - 1 : half;
+      }
+      calib[e + lo] = __uint_as_float(bits_of_key(key));
+    } else {
+      const int j = e - n;
+      const uint32_t key = nk[j];
+      int lo = 0, len = n;  // number of old keys <= key
+      while (len > 0) {
+        const int half = len >> 1;
+        const bool le = ok[lo + half] <= key;
+        lo = le ? lo + half + 1 : lo;
+        len = le ? len - half - 1 : half;
+      }
+      calib[j + lo] = __uint_as_float(bits_of_key(key));
+    }
+  }
+}
+
 }  // namespace atts

@@ -134,7 +134,8 @@ def test_classify_boundary_cases_and_no_counts():
 
 @pytest.mark.parametrize("n,k", [(0, 1), (0, 300), (1, 1), (256, 8), (4096, 64), (1000, 4097), (65536, 4096),
                                   (323584, 4096), (5000, 16384), (100, 40000), (7, 0),
-                                  (602112, 4096), (602113, 4096), (700000, 100), (20, 16385)])
+                                  (602112, 4096), (602113, 4096), (700000, 100), (20, 16385),
+                                  (20000, 1000), (28672, 3000), (28673, 10), (28000, 4096), (5, 8)])
 def test_calib_update_bit_exact(n, k):
     calib = np.sort(inputs.lognormal_scores(300 + n, n))
     new = inputs.lognormal_scores(400 + k, k)
@@ -180,6 +181,22 @@ def test_calib_update_duplicates_and_special_values():
     # a second insert on top of a buffer that already holds NaNs
     buf2, n3 = gpu_update(buf[:n2], new, n2 + new.size)
     assert np.array_equal(f32_bits(buf2[:n3]), f32_bits(orc.calib_update(buf[:n2], new)))
+
+
+def test_calib_update_small_in_place_path_special_values():
+    # few new scores into a small buffer: the single-block in-place kernel; ties, zeros, infinities, NaNs
+    calib = orc.calib_update(np.zeros(0, np.float32), np.concatenate(
+        [np.round(inputs.lognormal_scores(1, 2000), 1), np.array([np.nan, np.inf, -np.inf, -0.0], np.float32)]))
+    weird_nan = np.array([0x7F800001, 0xFFC00123], np.uint32).view(np.float32)
+    new = np.concatenate([np.round(inputs.lognormal_scores(2, 40), 1),
+                          np.array([-0.0, 0.0, np.inf, -np.inf, 3.0, 3.0], np.float32), weird_nan])
+    buf, n2 = gpu_update(calib, new, calib.size + new.size + 3)
+    assert np.array_equal(f32_bits(buf[:n2]), f32_bits(orc.calib_update(calib, new)))
+    assert np.all(f32_bits(buf[n2:]) == 0xFFFFFFFF)
+    # a non-canonical old buffer (-0.0 stored) is canonicalised on the way
+    old = np.array([-1.0, -0.0, 0.0, 2.0], np.float32)
+    buf, n2 = gpu_update(old, np.array([1.0], np.float32), 5)
+    assert np.array_equal(f32_bits(buf[:n2]), f32_bits(orc.calib_update(old, np.array([1.0], np.float32))))
 
 
 def test_calib_update_capacity_error_leaves_buffer_untouched():
