@@ -9,10 +9,12 @@
  *   - Pointers marked "dev" are device pointers of the current CUDA device, "host" are host
  *     pointers.  The caller owns every buffer, workspaces included; the library allocates no
  *     device memory and keeps no state between calls except a per-process cache of the device's
- *     properties and one device-side status word.
+ *     properties, one device-side status word and the fixed scratch of atts_calib_update_static.
  *   - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
- *     legacy default stream) and returns; results are valid in stream order.  The only call that
- *     synchronises is atts_last_device_status.
+ *     legacy default stream) and returns; results are valid in stream order, and a sequence of
+ *     calls can be captured in a CUDA graph once each entry point has been called once on the
+ *     device (the first call probes the device).  The only calls that synchronise are
+ *     atts_last_device_status and atts_profile_end.
  *   - The return value is an atts_status.  Argument errors are found before anything is launched
  *     and leave every output untouched.  There is no CPU or non-sm_100 fallback: on another device
  *     the calls return ATTS_ERR_ARCH, without a device ATTS_ERR_CUDA.

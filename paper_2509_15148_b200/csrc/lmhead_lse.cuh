@@ -1,9 +1,9 @@
 // Fused LM-head projection + online log-sum-exp + gather of the draft token's logit (sm_100a).
 //
-// logits[i, v] = sum_k H[i, k] * W[v, k] are produced in 128 x 256 tiles by tcgen05.mma (bf16 in,
-// fp32 accumulators in tensor memory), read back with tcgen05.ld and reduced per row to a running
-// (max, sum of exponentials); the logit of the row's own token is picked out on the way.  Logits
-// never leave the SM.  A second, tiny kernel merges the per-chunk partials into token log-probs,
+// logits[i, v] = sum_k H[i, k] * W[v, k] are produced in 128 x 256 tiles per CTA (256 x 256 per CTA pair)
+// by tcgen05.mma (bf16 in, fp32 accumulators in tensor memory), read back with tcgen05.ld and reduced
+// per row to a running (max, sum of exponentials); the logit of the row's own token is picked out on the
+// way.  Logits never leave the SM.  A second, tiny kernel merges the per-chunk partials into token log-probs,
 // a third reduces them per sample.
 #pragma once
 #include <cuda.h>
