@@ -250,3 +250,34 @@ def test_conformal_stress_sequence_bit_exact():
         assert n == calib.size
         assert np.array_equal(f32_bits(buf[:n]), f32_bits(calib))
     assert binding.last_device_status() == 0
+
+
+def test_randomised_sizes_and_value_mixes():
+    """Thirty random problems: random sizes around the kernels' mode switches, values rounded to force ties,
+    a sprinkling of special values; every output compared with the oracle bit for bit."""
+    rng = np.random.default_rng(20240607)
+    pool = np.array([0.0, -0.0, np.inf, -np.inf, np.nan, 1e-38, -1e-38, 3.0], np.float32)
+    for case in range(30):
+        n = int(rng.choice([0, 1, 2, 255, 8190, 8191, 8192, 20000, 28672, 28673, 70001]))
+        k = int(rng.choice([0, 1, 7, 64, 500, 4096, 4097]))
+        Nc = int(rng.choice([1, 3, 4, 1000, 4095, 65535, 65536, 131072 + 5]))
+        digits = int(rng.choice([1, 3, 6]))
+        calib_raw = np.round(inputs.lognormal_scores(1000 + case, n), digits)
+        new = np.round(inputs.lognormal_scores(2000 + case, k), digits)
+        scores = np.round(inputs.lognormal_scores(3000 + case, Nc), digits)
+        for arr in (calib_raw, new, scores):
+            if arr.size >= 4 and rng.random() < 0.5:
+                idx = rng.choice(arr.size, size=min(arr.size, 6), replace=False)
+                arr[idx] = rng.choice(pool, size=idx.size)
+        calib = orc.calib_update(np.zeros(0, np.float32), calib_raw)
+        numer, p = gpu_rank(scores, calib)
+        want = orc.conformal_numer_sorted(scores, calib)
+        assert np.array_equal(numer, want), (case, n, Nc)
+        assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want, n))), (case, n, Nc)
+        alpha = float(rng.choice([0.05, 0.1, 0.37, 0.5]))
+        stage, counts = gpu_classify(numer, n, alpha)
+        ws, wc = orc.classify(want, n, alpha)
+        assert np.array_equal(stage, ws) and np.array_equal(counts, wc), (case, n, Nc, alpha)
+        buf, n2 = gpu_update(calib, new, n + k + 2)
+        assert n2 == n + k
+        assert np.array_equal(f32_bits(buf[:n2]), f32_bits(orc.calib_update(calib, new))), (case, n, k)

@@ -198,3 +198,19 @@ def test_argument_errors_on_device():
     assert e.value.status == 6
     torch.cuda.synchronize()
     assert np.all(lp.cpu().numpy().view(np.uint32) == 0xFFFFFFFF)      # nothing was launched
+
+
+def test_randomised_shapes():
+    """A dozen random shapes (rows, hidden size, vocabulary, ragged samples) against the oracle."""
+    rng = np.random.default_rng(77)
+    for case in range(12):
+        M = int(rng.integers(1, 1500))
+        d = 64 * int(rng.integers(1, 12))
+        V = int(rng.integers(1, 7000))
+        S = int(rng.integers(1, 9))
+        cuts = np.sort(rng.integers(0, M + 1, size=S - 1))
+        off = np.concatenate([[0], cuts, [M]]).astype(np.int32)
+        Hb, Wb = inputs.hidden(500 + case, M, d), inputs.lm_head(600 + case, V, d)
+        ids = inputs.zipf_ids(700 + case, M, V)
+        ids[rng.integers(0, M)] = V - 1
+        check_against_oracle(Hb, Wb, ids, off, mode=int(rng.integers(0, 4)))
