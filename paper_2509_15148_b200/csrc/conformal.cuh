@@ -64,7 +64,7 @@ __device__ __forceinline__ void tree_descend(const float (&s)[4], const float* _
 }
 
 __device__ __forceinline__ void rank_four(const float (&s)[4], const float* __restrict__ sp, int P, int L,
-                                          const float* __restrict__ calib, int n, uint32_t (&numer)[4]) {
+                                          const float* __restrict__ calib, int n, bool vec8, uint32_t (&numer)[4]) {
   int cnt[4];
   switch (P) {  // the descent is unrolled for every table depth
     case 1: tree_descend<1>(s, sp, cnt); break;
@@ -91,7 +91,10 @@ __device__ __forceinline__ void rank_four(const float (&s)[4], const float* __re
     int base[4], pos[4] = {0, 0, 0, 0};
 #pragma unroll
     for (int e = 0; e < 4; ++e) base[e] = cnt[e] ? ((cnt[e] - 1) << L) + 1 : n;
-    for (int step = 1 << (L - 1); step > 0; step >>= 1) {
+    // With vec8 (L >= 3 and a 32-byte aligned buffer) the binary steps stop at windows of 7 entries; those
+    // 7 and the entry before them are one aligned 32-byte group, fetched with a single 256-bit load.
+    const int last_step = vec8 ? 8 : 1;
+    for (int step = 1 << (L - 1); step >= last_step; step >>= 1) {
       float v[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -100,6 +103,26 @@ __device__ __forceinline__ void rank_four(const float (&s)[4], const float* __re
       }
 #pragma unroll
       for (int e = 0; e < 4; ++e) pos[e] += (v[e] < s[e]) ? step : 0;
+    }
+    if (vec8) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int g0 = base[e] + pos[e] - 1;  // multiple of 8; entries g0 + 1 .. g0 + 7 are the window
+        int c = 0;
+        if (cnt[e] != 0) {
+          if (g0 + 8 <= n) {
+            float w[8];
+            asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=f"(w[0]), "=f"(w[1]), "=f"(w[2]), "=f"(w[3]), "=f"(w[4]), "=f"(w[5]), "=f"(w[6]), "=f"(w[7])
+                         : "l"(calib + g0));
+#pragma unroll
+            for (int i = 1; i < 8; ++i) c += (w[i] < s[e]) ? 1 : 0;
+          } else {
+            for (int i = 1; i < 8 && g0 + i < n; ++i) c += (__ldg(calib + g0 + i) < s[e]) ? 1 : 0;
+          }
+        }
+        pos[e] += c;
+      }
     }
 #pragma unroll
     for (int e = 0; e < 4; ++e) below[e] = cnt[e] ? base[e] + pos[e] : 0;
@@ -147,6 +170,7 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
   __syncthreads();
   const float denom = (float)(n + 1);
   const float qnan = __uint_as_float(0x7FC00000u);
+  const bool vec8 = L >= 3 && (reinterpret_cast<uintptr_t>(calib) & 31u) == 0;
   const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
   for (int64_t base = (int64_t)blockIdx.x * per_block; base < Nc; base += (int64_t)gridDim.x * per_block) {
     const int64_t j = base + (int64_t)threadIdx.x * kRankPerThread;
@@ -161,7 +185,7 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
 #pragma unroll
       for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
     }
-    rank_four(s, sp, P, L, calib, n, r);
+    rank_four(s, sp, P, L, calib, n, vec8, r);
     float p[4];
     if (tabulated) {
 #pragma unroll

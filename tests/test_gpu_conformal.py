@@ -95,6 +95,21 @@ def test_rank_many_candidates_tied_clustered_and_special_data(n):
         assert np.array_equal(numer[idx], orc.conformal_numer_count(scores[idx], calib)), name
 
 
+def test_rank_buffer_not_32_byte_aligned():
+    # the kernel's 256-bit loads need a 32-byte aligned buffer; any other 4-byte aligned pointer takes the scalar path
+    n, Nc = 100000, 1 << 17
+    calib = np.sort(inputs.lognormal_scores(31, n))
+    scores = inputs.lognormal_scores(32, Nc)
+    want = orc.conformal_numer_sorted(scores, calib)
+    for shift in (0, 1, 3, 8):
+        buf = torch.empty(n + 16, device="cuda")
+        buf[shift:shift + n] = dev(calib)
+        numer = poison((Nc,), torch.int32)
+        binding.conformal_rank(dev(scores), buf[shift:], n, numer, None)
+        torch.cuda.synchronize()
+        assert np.array_equal(host_u32(numer), want), shift
+
+
 def test_rank_without_pvalue_output_and_empty_input():
     calib = np.sort(inputs.lognormal_scores(5, 300))
     scores = inputs.lognormal_scores(6, 77)
