@@ -352,7 +352,7 @@ sort_new_kernel(const float* __restrict__ new_scores, int k, uint32_t* __restric
 //   old[i]  -> slot i + #{new <  old[i]}
 //   new[j]  -> slot j + #{old <= new[j]}
 // written to `out` (n + k entries).  The new keys sit in shared memory for the first search; the
-// second searches the old buffer in global memory.
+// second searches the old buffer in global memory, 32 probes at a time.
 // ---------------------------------------------------------------------------------------------
 constexpr int kMergeThreads = 512;
 
@@ -362,31 +362,39 @@ merge_kernel(const float* __restrict__ old_buf, int n, const uint32_t* __restric
   extern __shared__ uint32_t nk[];
   for (int t = threadIdx.x; t < k; t += kMergeThreads) nk[t] = new_keys[t];
   __syncthreads();
-  const int total = n + k;
-  for (int e = blockIdx.x * kMergeThreads + threadIdx.x; e < total; e += gridDim.x * kMergeThreads) {
-    if (e < n) {
-      uint32_t bits = canonical_bits(old_buf[e]);
-      uint32_t key = key_of_bits(bits);
-      int lo = 0, len = k;  // number of new keys < key
-      while (len > 0) {
-        int half = len >> 1;
-        bool less = nk[lo + half] < key;
-        lo = less ? lo + half + 1 : lo;
-        len = less ? len - half - 1 : half;
-      }
-      out[e + lo] = __uint_as_float(bits);
-    } else {
-      int j = e - n;
-      uint32_t key = nk[j];
-      int lo = 0, len = n;  // number of old keys <= key
-      while (len > 0) {
-        int half = len >> 1;
-        bool le = key_of_bits(canonical_bits(__ldg(old_buf + lo + half))) <= key;
-        lo = le ? lo + half + 1 : lo;
-        len = le ? len - half - 1 : half;
-      }
-      out[j + lo] = __uint_as_float(bits_of_key(key));
+  // New keys first, one warp each: a 32-way search of the old buffer (every lane probes one of 32 evenly spaced
+  // entries, a ballot keeps the interval between the last "<=" and the first ">"), so the chain of dependent
+  // loads is log32(n) long instead of log2(n) and overlaps the bulk work below.
+  const int lane = threadIdx.x & 31;
+  const int warps_per_block = kMergeThreads / 32;
+  for (int j = blockIdx.x * warps_per_block + (threadIdx.x >> 5); j < k; j += gridDim.x * warps_per_block) {
+    const uint32_t key = nk[j];
+    int lo = 0, hi = n;  // the number of old keys <= key lies in [lo, hi]
+    while (hi > lo) {
+      const int width = hi - lo;
+      const int p = width >= 32 ? lo + (int)(((long long)width * (lane + 1)) >> 5) - 1 : lo + lane;
+      const bool le = p < hi && key_of_bits(canonical_bits(__ldg(old_buf + p))) <= key;
+      const int c = __popc(__ballot_sync(0xFFFFFFFFu, le));  // the predicate is true on a prefix of the lanes
+      const int p_prev = __shfl_sync(0xFFFFFFFFu, p, c > 0 ? c - 1 : 0);
+      const int p_next = __shfl_sync(0xFFFFFFFFu, p, c < 32 ? c : 31);
+      const int probes = width >= 32 ? 32 : width;
+      if (c > 0) lo = p_prev + 1;
+      if (c < probes) hi = p_next;
     }
+    if (lane == 0) out[j + lo] = __uint_as_float(bits_of_key(key));
+  }
+  // Old entries: each searches the sorted new keys in shared memory.
+  for (int e = blockIdx.x * kMergeThreads + threadIdx.x; e < n; e += gridDim.x * kMergeThreads) {
+    const uint32_t bits = canonical_bits(old_buf[e]);
+    const uint32_t key = key_of_bits(bits);
+    int lo = 0, len = k;  // number of new keys < key
+    while (len > 0) {
+      const int half = len >> 1;
+      const bool less = nk[lo + half] < key;
+      lo = less ? lo + half + 1 : lo;
+      len = less ? len - half - 1 : half;
+    }
+    out[e + lo] = __uint_as_float(bits);
   }
 }
 
