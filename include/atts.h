@@ -85,7 +85,7 @@ int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_
  *                      yields NaN for that row
  *   seg_offsets   dev  [S + 1] int32, 0 = o_0 <= o_1 <= ... <= o_S = M (not checked on the device
  *                      beyond clamping to [0, M])
- *   M, d, V, S         0 <= M < 2^31, d a multiple of 64 with 64 <= d <= 16384 (the fp32 accumulation error of
+ *   M, d, V, S         0 <= M <= 2^30, d a multiple of 64 with 64 <= d <= 16384 (the fp32 accumulation error of
  *                      a logit grows with d; 2e-3 on the log-probs was verified up to this size), 1 <= V < 2^31,
  *                      0 <= S
  *   token_logprob dev  [M] fp32 out, may be NULL

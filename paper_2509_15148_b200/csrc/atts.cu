@@ -140,7 +140,7 @@ static ScorePlan choose_score_plan(const DeviceInfo* di, int64_t M, int64_t d, i
 }
 
 static int check_score_shape(int64_t M, int64_t d, int64_t V, int64_t S) {
-  if (M < 0 || M >= (1ll << 31) - kBlockM || S < 0 || S >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  if (M < 0 || M > (1ll << 30) || S < 0 || S >= (1ll << 31)) return ATTS_ERR_SHAPE;
   if (d < 64 || d > 16384 || d % 64 != 0) return ATTS_ERR_SHAPE;
   if (V < 1 || V >= (1ll << 31) - kBlockN) return ATTS_ERR_SHAPE;
   return ATTS_OK;
@@ -309,7 +309,7 @@ int atts_score_logprob_scaled(const void* hidden_bf16, const void* lm_head_bf16,
 }
 
 int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float* row_scale, void* cuda_stream) {
-  if (M < 0 || M >= (1ll << 31) - kBlockM || d < 8 || d > 16384 || d % 8 != 0) return ATTS_ERR_SHAPE;
+  if (M < 0 || M > (1ll << 30) || d < 8 || d > 16384 || d % 8 != 0) return ATTS_ERR_SHAPE;
   if (!(eps >= 0.f)) return ATTS_ERR_ARG;
   if (M > 0 && (!hidden_bf16 || !row_scale)) return ATTS_ERR_NULL;
   if (!aligned(hidden_bf16, 16) || !aligned(row_scale, 4)) return ATTS_ERR_ALIGN;
