@@ -116,6 +116,27 @@ int atts_score_logprob_scaled(const void* hidden_bf16, const void* lm_head_bf16,
                               void* cuda_stream);
 
 /*
+ * Scoring with the vocabulary sharded over GPUs (W split by rows, as a tensor-parallel LM head is).  Each
+ * rank runs atts_score_slice on its rows of W and gets, per scored token, the triple
+ *   slice_stats[i] = { max_v z_iv,  sum_v exp(z_iv - max),  z_i[token_ids[i]] or -inf if that id is not in
+ *                      [vocab_offset, vocab_offset + V_slice) }
+ * over its slice (same fused kernel, logits never stored).  The ranks exchange their [M, 3] blocks (an
+ * all-gather of 12 bytes per token; this library does not communicate), and atts_score_combine merges G
+ * blocks laid out [G][M][3] into token log-probs and sample scores exactly as atts_score_logprob merges
+ * its own vocabulary chunks: LSE = Mx + log sum_g l_g exp(m_g - Mx).  A token id that no slice holds sets
+ * ATTS_DEV_TOKEN_ID_RANGE and yields NaN.
+ *   workspace of atts_score_slice: atts_score_workspace_bytes(M, d, V_slice, 0);
+ *   workspace of atts_score_combine: at least 4 * M + 512 bytes, 256-byte aligned.
+ * Other arguments as atts_score_logprob.
+ */
+int atts_score_slice(const void* hidden_bf16, const void* lm_head_slice_bf16, const int32_t* token_ids,
+                     int64_t M, int64_t d, int64_t V_slice, int64_t vocab_offset, float* slice_stats,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+int atts_score_combine(const float* slice_stats, int64_t G, const int32_t* seg_offsets, int64_t M, int64_t S,
+                       int32_t score_mode, float* token_logprob, float* sample_score, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream);
+
+/*
  * row_scale[i] = 1 / sqrt(mean_k hidden[i, k]^2 + eps), fp32 accumulation.
  *   hidden_bf16   dev  [M, d] bf16 row-major, 16-byte aligned, d a multiple of 8;  eps >= 0
  *   row_scale     dev  [M] fp32 out

@@ -19,7 +19,7 @@ EXPORTS = (
     "atts_last_device_status", "atts_profile_begin", "atts_profile_end",
     "atts_calib_update_static", "atts_rank_classify", "atts_score_logprob_scaled", "atts_rms_inv",
     "atts_threshold", "atts_classify_threshold", "atts_conformal_rank_conditional", "atts_classify_conditional",
-    "atts_debug_score_plan", "atts_debug_score_unit",
+    "atts_debug_score_plan", "atts_debug_score_unit", "atts_score_slice", "atts_score_combine",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -61,6 +61,10 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
                                        c_void_p, c_void_p, c_void_p]
     lib.atts_score_logprob_scaled.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64,
                                               c_int64, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.atts_score_slice.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int64, c_void_p, c_void_p,
+                                     c_size_t, c_void_p]
+    lib.atts_score_combine.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_int64, c_int32, c_void_p, c_void_p, c_void_p,
+                                       c_size_t, c_void_p]
     lib.atts_rms_inv.argtypes = [c_void_p, c_int64, c_int64, ctypes.c_float, c_void_p, c_void_p]
     lib.atts_threshold.argtypes = [c_void_p, c_int64, c_double, c_void_p, c_void_p]
     lib.atts_classify_threshold.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -133,6 +137,23 @@ def score_logprob_scaled(hidden, lm_head, token_ids, row_scale, seg_offsets, tok
                                             _ptr(sample_score), _ptr(workspace),
                                             workspace.numel() * workspace.element_size(), _stream()),
            "atts_score_logprob_scaled")
+
+
+def score_slice(hidden, lm_head_slice, token_ids, vocab_offset: int, slice_stats, workspace) -> None:
+    """Per-token (max, sum exp, token logit or -inf) over one vocabulary slice: slice_stats [M, 3] f32."""
+    M, d = hidden.shape
+    _check(load().atts_score_slice(_ptr(hidden), _ptr(lm_head_slice), _ptr(token_ids), M, d, lm_head_slice.shape[0],
+                                   int(vocab_offset), _ptr(slice_stats), _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream()), "atts_score_slice")
+
+
+def score_combine(slice_stats, seg_offsets, token_logprob, sample_score, workspace, score_mode: int = 0) -> None:
+    """Merge slice_stats [G, M, 3] (all ranks' blocks in rank order) into token log-probs and sample scores."""
+    G, M = slice_stats.shape[0], slice_stats.shape[1]
+    S = seg_offsets.numel() - 1
+    _check(load().atts_score_combine(_ptr(slice_stats), G, _ptr(seg_offsets), M, S, score_mode, _ptr(token_logprob),
+                                     _ptr(sample_score), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                     _stream()), "atts_score_combine")
 
 
 def rms_inv(hidden, eps: float, row_scale) -> None:

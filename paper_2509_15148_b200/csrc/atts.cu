@@ -221,14 +221,17 @@ int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_
   return ATTS_OK;
 }
 
+// slice_stats != nullptr: W is the vocabulary slice starting at id vocab_offset; the call stops after writing one
+// (max, sum, token logit) triple per row (no log-probs, no scores).
 static int score_impl(const void* hidden_bf16, const void* lm_head_bf16, const int32_t* token_ids,
                       const float* row_scale, const int32_t* seg_offsets, int64_t M, int64_t d, int64_t V, int64_t S,
                       int32_t score_mode, float* token_logprob, float* sample_score, void* workspace,
-                      size_t workspace_bytes, void* cuda_stream) {
+                      size_t workspace_bytes, void* cuda_stream, int64_t vocab_offset = 0,
+                      float* slice_stats = nullptr) {
   int st = check_score_shape(M, d, V, S);
   if (st != ATTS_OK) return st;
   if (score_mode < 0 || score_mode > 3) return ATTS_ERR_ARG;
-  if (!lm_head_bf16 || !seg_offsets || !workspace) return ATTS_ERR_NULL;
+  if (!lm_head_bf16 || (!seg_offsets && !slice_stats) || !workspace) return ATTS_ERR_NULL;
   if (M > 0 && (!hidden_bf16 || !token_ids)) return ATTS_ERR_NULL;
   if (S > 0 && !sample_score) return ATTS_ERR_NULL;
   if (!aligned(hidden_bf16, 16) || !aligned(lm_head_bf16, 16) || !aligned(workspace, 256) ||
@@ -238,7 +241,8 @@ static int score_impl(const void* hidden_bf16, const void* lm_head_bf16, const i
   const DeviceInfo* di;
   st = device_info(&di);
   if (st != ATTS_OK) return st;
-  const ScorePlan plan = choose_score_plan(di, M, d, V);
+  ScorePlan plan = choose_score_plan(di, M, d, V);
+  plan.vocab_offset = (int)vocab_offset;
   const ScoreWs ws = score_ws(plan);
   if (workspace_bytes < ws.total) return ATTS_ERR_WORKSPACE;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -279,6 +283,11 @@ static int score_impl(const void* hidden_bf16, const void* lm_head_bf16, const i
     }
     if (timed) cudaEventRecord(g_prof.ev[2 * g_prof.used++ + 1], stream);
     if ((st = launch_status()) != ATTS_OK) return st;
+    if (slice_stats) {
+      slice_stats_kernel<<<(unsigned)((M + 255) / 256), 256, 0, stream>>>(partial, gathered, token_ids, (int)M, plan.M_pad,
+                                                                          plan.C, (int)V, (int)vocab_offset, slice_stats);
+      return launch_status();
+    }
     lse_combine_kernel<<<(unsigned)((M + 255) / 256), 256, 0, stream>>>(partial, gathered, token_ids, (int)M, plan.M_pad,
                                                                         plan.C, (int)V, logprob_ws, token_logprob,
                                                                         di->dev_status);
@@ -306,6 +315,44 @@ int atts_score_logprob_scaled(const void* hidden_bf16, const void* lm_head_bf16,
   if (M > 0 && !row_scale) return ATTS_ERR_NULL;
   return score_impl(hidden_bf16, lm_head_bf16, token_ids, row_scale, seg_offsets, M, d, V, S, score_mode, token_logprob,
                     sample_score, workspace, workspace_bytes, cuda_stream);
+}
+
+int atts_score_slice(const void* hidden_bf16, const void* lm_head_slice_bf16, const int32_t* token_ids, int64_t M,
+                     int64_t d, int64_t V_slice, int64_t vocab_offset, float* slice_stats, void* workspace,
+                     size_t workspace_bytes, void* cuda_stream) {
+  if (vocab_offset < 0 || vocab_offset >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  if (M > 0 && !slice_stats) return ATTS_ERR_NULL;
+  if (!aligned(slice_stats, 4)) return ATTS_ERR_ALIGN;
+  if (M == 0) return check_score_shape(M, d, V_slice, 0);
+  return score_impl(hidden_bf16, lm_head_slice_bf16, token_ids, nullptr, nullptr, M, d, V_slice, 0, 0, nullptr, nullptr,
+                    workspace, workspace_bytes, cuda_stream, vocab_offset, slice_stats);
+}
+
+int atts_score_combine(const float* slice_stats, int64_t G, const int32_t* seg_offsets, int64_t M, int64_t S,
+                       int32_t score_mode, float* token_logprob, float* sample_score, void* workspace,
+                       size_t workspace_bytes, void* cuda_stream) {
+  if (M < 0 || M > (1ll << 30) || S < 0 || S >= (1ll << 31) || G < 1 || G > 1024) return ATTS_ERR_SHAPE;
+  if (score_mode < 0 || score_mode > 3) return ATTS_ERR_ARG;
+  if (!seg_offsets || !workspace || (M > 0 && !slice_stats) || (S > 0 && !sample_score)) return ATTS_ERR_NULL;
+  if (!aligned(slice_stats, 4) || !aligned(seg_offsets, 4) || !aligned(token_logprob, 4) || !aligned(sample_score, 4) ||
+      !aligned(workspace, 256))
+    return ATTS_ERR_ALIGN;
+  if (workspace_bytes < round_up((size_t)M * 4, 256) + 256) return ATTS_ERR_WORKSPACE;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  float* logprob_ws = static_cast<float*>(workspace);
+  if (M > 0) {
+    stats_combine_kernel<<<(unsigned)((M + 255) / 256), 256, 0, stream>>>(slice_stats, (int)G, (int)M, logprob_ws,
+                                                                          token_logprob, di->dev_status);
+    if ((st = launch_status()) != ATTS_OK) return st;
+  }
+  if (S > 0) {
+    segment_score_kernel<<<(unsigned)S, 256, 0, stream>>>(logprob_ws, seg_offsets, (int)M, (int)S, score_mode, sample_score);
+    if ((st = launch_status()) != ATTS_OK) return st;
+  }
+  return ATTS_OK;
 }
 
 int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float* row_scale, void* cuda_stream) {

@@ -52,6 +52,7 @@ struct ScorePlan {
   int units;   // RB * C
   int M_pad;   // RB * rows per unit
   int ctas;    // 1 or 2: CTAs per worker
+  int vocab_offset;  // id of this W's first row (0 unless W is a slice of a sharded vocabulary)
 };
 
 __host__ __device__ inline void decode_unit(const ScorePlan& p, int u, int& rb, int& c, int& nt0, int& nt1) {
@@ -389,7 +390,9 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
       int rb, c, nt0, nt1;
       decode_unit(plan, u, rb, c, nt0, nt1);
       const int row = rb * Cfg::kRowsPerUnit + (int)rank * kBlockM + quarter * 32 + lane;
-      const int y = (row < plan.M) ? token_ids[row] : -1;
+      // the token's column in this W; ids outside [0, V) (another vocabulary slice, or invalid) never match
+      int y = (row < plan.M) ? token_ids[row] - plan.vocab_offset : -1;
+      if (y >= plan.V) y = -1;
       // optional per-row factor on the logits (finite, > 0): folded into the exponent's scale, so it costs nothing per
       // element; the running maximum is kept on the unscaled logits
       const float rs = (row_scale != nullptr && row < plan.M) ? row_scale[row] : 1.f;
@@ -516,6 +519,57 @@ lse_combine_kernel(const float2* __restrict__ partial, const float* __restrict__
     atomicOr(dev_status, 1u);
   } else {
     lp = gathered[row] - (mx + logf(sum));
+  }
+  logprob_ws[row] = lp;
+  if (logprob_out) logprob_out[row] = lp;
+}
+
+// ------------------------------------------------------------------------------------------
+// Vocabulary sharding (W split by rows over GPUs).  A slice's chunk partials are reduced to one triple per
+// row, stats[row] = (max z, sum exp(z - max), z[token] or -inf if the token lies in another slice); after the
+// ranks have exchanged their triples, G triples per row are merged exactly as chunk partials are.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+slice_stats_kernel(const float2* __restrict__ partial, const float* __restrict__ gathered,
+                   const int32_t* __restrict__ token_ids, int M, int M_pad, int C, int V, int vocab_offset,
+                   float* __restrict__ stats) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= M) return;
+  float mx = -INFINITY;
+  for (int c = 0; c < C; ++c) mx = fmaxf(mx, partial[(size_t)c * M_pad + row].x);
+  float sum = 0.f;
+  for (int c = 0; c < C; ++c) {
+    const float2 p = partial[(size_t)c * M_pad + row];
+    sum += p.y * expf(p.x - mx);
+  }
+  const int y = token_ids[row] - vocab_offset;
+  stats[3 * (size_t)row + 0] = mx;
+  stats[3 * (size_t)row + 1] = sum;
+  stats[3 * (size_t)row + 2] = (y >= 0 && y < V) ? gathered[row] : -INFINITY;
+}
+
+__global__ void __launch_bounds__(256)
+stats_combine_kernel(const float* __restrict__ stats, int G, int M, float* __restrict__ logprob_ws,
+                     float* __restrict__ logprob_out, unsigned int* __restrict__ dev_status) {
+  const int row = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= M) return;
+  float mx = -INFINITY, g = -INFINITY;
+  for (int s = 0; s < G; ++s) {
+    const float* t = stats + 3 * ((size_t)s * M + row);
+    mx = fmaxf(mx, t[0]);
+    g = fmaxf(g, t[2]);
+  }
+  float sum = 0.f;
+  for (int s = 0; s < G; ++s) {
+    const float* t = stats + 3 * ((size_t)s * M + row);
+    sum += t[1] * expf(t[0] - mx);
+  }
+  float lp;
+  if (g == -INFINITY) {  // no slice held the token: id out of range
+    lp = __uint_as_float(0x7FC00000u);
+    atomicOr(dev_status, 1u);
+  } else {
+    lp = g - (mx + logf(sum));
   }
   logprob_ws[row] = lp;
   if (logprob_out) logprob_out[row] = lp;

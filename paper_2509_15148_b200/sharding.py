@@ -30,3 +30,24 @@ def all_gather_scores(local_scores, world: int, dist=None):
     parts = [torch.empty_like(local_scores) for _ in range(world)]
     dist.all_gather(parts, local_scores.contiguous())
     return torch.cat(parts)
+
+
+def vocab_range(V: int, world: int, rank: int, align: int = 256) -> tuple[int, int]:
+    """Rows [begin, end) of the LM head that `rank` holds when the vocabulary is sharded: equal slices rounded up
+    to a multiple of `align` rows (one vocabulary tile), the last rank taking what is left (possibly nothing)."""
+    if not (0 <= rank < world):
+        raise ValueError("rank out of range")
+    per = -(-V // world)
+    per = -(-per // align) * align
+    begin = min(rank * per, V)
+    return begin, min(begin + per, V)
+
+
+def all_gather_slice_stats(local_stats, world: int, dist=None):
+    """[M, 3] per rank -> [world, M, 3] in rank order (the layout atts_score_combine reads)."""
+    import torch
+    if world == 1:
+        return local_stats.unsqueeze(0)
+    parts = [torch.empty_like(local_stats) for _ in range(world)]
+    dist.all_gather(parts, local_stats.contiguous())
+    return torch.stack(parts)

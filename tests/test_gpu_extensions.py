@@ -108,3 +108,41 @@ def test_rms_inv_and_scaled_scoring(M, d, V):
     binding.score_logprob(H, dev_bf16(Wb), dev(ids), dev(off), lp2, sc, ws)
     torch.cuda.synchronize()
     assert torch.equal(lp1, lp2)
+
+
+@pytest.mark.parametrize("M,d,V,cuts", [(300, 192, 5000, (0, 1700, 1701, 5000)), (1000, 256, 4096, (0, 1024, 2048, 3072, 4096)),
+                                        (130, 64, 600, (0, 600)), (4096, 1024, 30000, (0, 9999, 20480, 30000))])
+def test_vocabulary_sliced_scoring_equals_the_full_definition(M, d, V, cuts):
+    """W split by rows into G slices (as on G tensor-parallel ranks), each scored on its own, the [M, 3] blocks
+    stacked in rank order and merged: the result is the log-softmax over the whole vocabulary."""
+    Hb, Wb = inputs.hidden(1, M, d), inputs.lm_head(2, V, d)
+    ids = inputs.zipf_ids(3, M, V)
+    ids[:6] = np.array([0, cuts[1] - 1, cuts[1] % V, V - 1, cuts[-2], cuts[-2] - 1 if cuts[-2] > 0 else 0], np.int32)
+    off = np.array([0, M // 3, M], np.int32)
+    H, idd = dev_bf16(Hb), dev(ids)
+    G = len(cuts) - 1
+    stats = poison((G, M, 3), torch.float32)
+    for g in range(G):
+        a, b = cuts[g], cuts[g + 1]
+        Wg = dev_bf16(Wb[a:b])
+        ws = workspace(binding.score_workspace_bytes(M, d, b - a, 0))
+        binding.score_slice(H, Wg, idd, a, stats[g], ws)
+    lp = poison((M,), torch.float32)
+    sc = poison((2,), torch.float32)
+    binding.score_combine(stats, dev(off), lp, sc, workspace(4 * M + 512))
+    assert binding.last_device_status() == 0
+    want = orc.token_logprob(Hb, Wb, ids)
+    assert np.abs(lp.cpu().numpy() - want).max() <= 2e-3
+    assert np.abs(sc.cpu().numpy() - orc.sample_score(want, off)).max() <= 2e-3
+    # exactly one slice holds each token's logit
+    held = torch.isfinite(stats[:, :, 2]).sum(dim=0).cpu().numpy()
+    assert (held == 1).all()
+    # an id beyond every slice is flagged and gives NaN
+    bad = ids.copy()
+    bad[7] = V
+    for g in range(G):
+        a, b = cuts[g], cuts[g + 1]
+        binding.score_slice(H, dev_bf16(Wb[a:b]), dev(bad), a, stats[g], workspace(binding.score_workspace_bytes(M, d, b - a, 0)))
+    binding.score_combine(stats, dev(off), lp, sc, workspace(4 * M + 512))
+    assert binding.last_device_status() & binding.DEV_TOKEN_ID_RANGE
+    assert np.isnan(lp.cpu().numpy()[7])

@@ -63,3 +63,47 @@ def test_two_ranks_keep_identical_buffers(tmp_path):
     assert np.array_equal(bufs[0].view(np.uint32), calib.view(np.uint32))
     for r in range(world):
         assert np.array_equal(np.load(tmp_path / f"stage_{r}.npy"), np.concatenate(want_stage[r]))
+
+
+def test_vocab_range_partitions_the_vocabulary():
+    for V in (1, 255, 256, 257, 8192, 152064, 128256):
+        for world in (1, 2, 3, 8):
+            spans = [sharding.vocab_range(V, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == V
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            assert all(a % 256 == 0 for a, _ in spans if a < V)
+
+
+def _vocab_worker(rank: int, world: int, port: int, out_dir: str):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    M, d, V = 40, 32, 700
+    Hb, Wb = inputs.hidden(1, M, d), inputs.lm_head(2, V, d)
+    ids = inputs.zipf_ids(3, M, V)
+    a, b = sharding.vocab_range(V, world, rank)
+    # this rank's triple per token over its slice of the vocabulary (float64 stand-in for atts_score_slice)
+    z = orc.logits(Hb, Wb[a:b]) if b > a else np.full((M, 0), -np.inf)
+    mx = z.max(axis=1) if b > a else np.full(M, -np.inf)
+    sm = np.exp(z - mx[:, None]).sum(axis=1) if b > a else np.zeros(M)
+    g = np.where((ids >= a) & (ids < b), z[np.arange(M), np.clip(ids - a, 0, max(b - a - 1, 0))] if b > a else -np.inf, -np.inf)
+    local = torch.from_numpy(np.stack([mx, sm, g], axis=1))
+    allst = sharding.all_gather_slice_stats(local, world, dist).numpy()          # [world, M, 3]
+    assert allst.shape == (world, M, 3)
+    Mx = allst[:, :, 0].max(axis=0)
+    lse = Mx + np.log((allst[:, :, 1] * np.exp(allst[:, :, 0] - Mx)).sum(axis=0))
+    lp = allst[:, :, 2].max(axis=0) - lse
+    np.save(os.path.join(out_dir, f"lp_{rank}.npy"), lp)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_two_ranks_vocabulary_sharded_scoring(tmp_path):
+    world = 2
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    mp.spawn(_vocab_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    want = orc.token_logprob(inputs.hidden(1, 40, 32), inputs.lm_head(2, 700, 32), inputs.zipf_ids(3, 40, 700))
+    for r in range(world):
+        np.testing.assert_allclose(np.load(tmp_path / f"lp_{r}.npy"), want, atol=1e-12)
