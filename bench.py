@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 KERNELS_PER_STEP = 6  # lmhead_lse, lse_combine, segment_score, rank, classify, small_update (n + k small: one block)
 # DRAM bytes per launch of the fused kernel on this workload, from an ncu capture (profiles/), valid only for
 # the kernel source it was taken on: (sha256 of csrc/lmhead_lse.cuh, dram__bytes_read.sum + dram__bytes_write.sum).
-K1_TRAFFIC = ("34531d2d4f3db0477e686364ea18f1b8468be08de5527365686012672ec649ee", 7.483e10)
+K1_TRAFFIC = ("18fa410ba28afbe3a4a16a57cdf0e525b99c7545f56f72480992126599fc958b", 5.255e10)
 
 
 def k1_traffic_bytes():
