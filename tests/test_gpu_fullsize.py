@@ -51,6 +51,52 @@ def test_full_shape_sampled_rows(name, scattered):
     means = -lp_h.astype(np.float64).reshape(N, T).mean(axis=1)
     assert np.abs(means - sc_h).max() <= 1e-5
 
+    # ---- the configuration's conformal step on the kernel's own fp32 scores, bit for bit against the oracle.
+    # The calibration buffer (n scores "from the same generator on another seed") is filled by scoring n / N
+    # calibration batches of the same distribution drawn on the device, through the same entry points.
+    n_cal, alphas = c["n"], c["alphas"]
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(inputs.BASE_SEED + 100)
+    W_d, off_d = dev_bf16(Wb), dev(off)
+    cdf = torch.cumsum(torch.arange(1, V + 1, device="cuda", dtype=torch.float64) ** -1.1, 0)
+    cdf /= cdf[-1].clone()
+    calib = poison((n_cal + N,), torch.float32)
+    ws_c = workspace(binding.calib_workspace_bytes(n_cal, N))
+    Hc = torch.empty((M, d), dtype=torch.bfloat16, device="cuda")
+    sc_c = poison((N,), torch.float32)
+    n_fill, cal_host = 0, np.zeros(0, np.float32)
+    for _ in range(n_cal // N):
+        for r0 in range(0, M, 8192):
+            x = torch.randn(min(8192, M - r0), d, device="cuda", generator=gen)
+            Hc[r0:r0 + x.shape[0]] = (x / x.pow(2).mean(1, keepdim=True).sqrt()).to(torch.bfloat16)
+        u = torch.rand(M, device="cuda", dtype=torch.float64, generator=gen)
+        idc = torch.searchsorted(cdf, u, right=True).clamp_(max=V - 1).to(torch.int32)
+        binding.score_logprob(Hc, W_d, idc, off_d, None, sc_c, ws)
+        n_fill = binding.calib_update(calib, n_fill, sc_c, ws_c)
+        cal_host = orc.calib_update(cal_host, sc_c.cpu().numpy())
+    assert n_fill == n_cal
+    assert np.array_equal(f32_bits(calib[:n_cal]), f32_bits(cal_host))
+    numer = poison((N,), torch.int32)
+    p = poison((N,), torch.float32)
+    stage = poison((N,), torch.uint8)
+    counts = poison((3,), torch.int32)
+    binding.conformal_rank(sc, calib, n_cal, numer, p)
+    want_numer = orc.conformal_numer_sorted(sc_h, cal_host)
+    assert np.array_equal(host_u32(numer), want_numer)
+    assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, n_cal)))
+    assert np.array_equal(want_numer, orc.conformal_numer_count(sc_h, cal_host))
+    for alpha in alphas:
+        binding.classify(numer, n_cal, alpha, stage, counts)
+        want_stage, want_counts = orc.classify(want_numer, n_cal, alpha)
+        assert np.array_equal(stage.cpu().numpy(), want_stage)
+        assert np.array_equal(host_u32(counts), want_counts)
+        # exchangeable test and calibration samples: the number taken over by the target is Binomial(N, ~alpha)
+        assert want_counts[2] <= alpha * N + 5 * np.sqrt(alpha * (1 - alpha) * N) + 1
+    n_after = binding.calib_update(calib, n_cal, sc, ws_c)
+    assert n_after == n_cal + N
+    assert np.array_equal(f32_bits(calib), f32_bits(orc.calib_update(cal_host, sc_h)))
+    assert binding.last_device_status() == 0
+
 
 def test_conformal_stress_at_maximum_buffer_size():
     """Last step of the conformal-only workload: 2^20 candidates against n = 323,584, three alphas, insert 4,096."""
