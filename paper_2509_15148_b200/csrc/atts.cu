@@ -81,6 +81,12 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaFuncSetAttribute(rank_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      const int bucket_smem = 4 * ((1 << kBucketMaxLog2) + 1 + 2 * kBucketMaxN + kBucketPad + 2);
+      ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       kSortMaxK * 4) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(small_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -372,6 +378,25 @@ int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float
 // Shared launcher of the rank kernel, with or without the fused thresholding.
 static int launch_rank(const DeviceInfo* di, const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
                        uint32_t* numer, float* pvalue, int n_alpha, const FusedClassify& fc, cudaStream_t stream) {
+  // Many candidates against a buffer that fits in shared memory: the bucket form (one table lookup and three
+  // probes per candidate instead of a log2(n)-step descent).  Its per-block set-up is only repaid by many candidates.
+  if (n >= 1 && n <= kBucketMaxN && Nc >= kBucketMinCandidates) {
+    int Blog2 = 10;
+    while (Blog2 < kBucketMaxLog2 && (1ll << Blog2) < 8 * n) ++Blog2;
+    const int64_t per_blk = (int64_t)kRankThreads * kRankPerThread;
+    int64_t nblk = (Nc + per_blk - 1) / per_blk;
+    if (nblk > di->sm_count) nblk = di->sm_count;
+    const dim3 g((unsigned)nblk), b(kRankThreads);
+    const size_t sm = 4 * (((size_t)1 << Blog2) + 1 + (size_t)n + kBucketPad + (pvalue ? (size_t)n + 2 : 0));
+    switch (n_alpha) {
+      case 0: rank_bucket_kernel<0><<<g, b, sm, stream>>>(scores, Nc, calib_sorted, (int)n, Blog2, numer, pvalue, fc); break;
+      case 1: rank_bucket_kernel<1><<<g, b, sm, stream>>>(scores, Nc, calib_sorted, (int)n, Blog2, numer, pvalue, fc); break;
+      case 2: rank_bucket_kernel<2><<<g, b, sm, stream>>>(scores, Nc, calib_sorted, (int)n, Blog2, numer, pvalue, fc); break;
+      case 3: rank_bucket_kernel<3><<<g, b, sm, stream>>>(scores, Nc, calib_sorted, (int)n, Blog2, numer, pvalue, fc); break;
+      default: rank_bucket_kernel<4><<<g, b, sm, stream>>>(scores, Nc, calib_sorted, (int)n, Blog2, numer, pvalue, fc); break;
+    }
+    return launch_status();
+  }
   // Table: the whole buffer when it has at most 8191 entries, else every 2^L-th entry.  Few candidates do
   // not repay a large strided table fill, so they get a smaller one.
   const int64_t max_slots = (Nc >= (1 << 16) ? (1 << kRankMaxTableLog2) : (1 << 10)) - 1;

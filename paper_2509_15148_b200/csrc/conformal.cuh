@@ -145,13 +145,80 @@ struct FusedClassify {
   uint32_t* counts;  // [NA][3] or nullptr
 };
 
+// Per-thread tallies of the fused thresholding, and the code both rank kernels share: writing the numerators,
+// p-values and stage bytes of four candidates, and the block's contribution to the stage counts.
+template <int NA>
+struct StageTally {
+  uint32_t c1[NA > 0 ? NA : 1] = {}, c3[NA > 0 ? NA : 1] = {}, seen = 0;
+};
+
+template <int NA>
+__device__ __forceinline__ void emit_four(int64_t j, int64_t Nc, bool full, const uint32_t (&r)[4], const float (&p)[4],
+                                          uint32_t* __restrict__ numer, float* __restrict__ pvalue,
+                                          const FusedClassify& fc, StageTally<NA>& tally) {
+  if (full) {
+    *reinterpret_cast<uint4*>(numer + j) = make_uint4(r[0], r[1], r[2], r[3]);
+    if (pvalue) *reinterpret_cast<float4*>(pvalue + j) = make_float4(p[0], p[1], p[2], p[3]);
+  } else {
+    for (int e = 0; e < 4 && j + e < Nc; ++e) {
+      numer[j + e] = r[e];
+      if (pvalue) pvalue[j + e] = p[e];
+    }
+  }
+  if (NA > 0) {
+    const int valid = full ? 4 : (int)(Nc - j);
+    tally.seen += (uint32_t)valid;
+#pragma unroll
+    for (int a = 0; a < NA; ++a) {
+      uint32_t st[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        st[e] = stage_of(r[e], fc.k_alpha[a]);
+        tally.c1[a] += (e < valid) && (st[e] == 1u);
+        tally.c3[a] += (e < valid) && (st[e] == 3u);
+      }
+      if (full) {
+        *reinterpret_cast<uint32_t*>(fc.stage[a] + j) = st[0] | (st[1] << 8) | (st[2] << 16) | (st[3] << 24);
+      } else {
+        for (int e = 0; e < valid; ++e) fc.stage[a][j + e] = (uint8_t)st[e];
+      }
+    }
+  }
+}
+
+// Adds the block's stage counts to fc.counts ([NA][3]); every thread of the block calls it.
+template <int NA>
+__device__ __forceinline__ void flush_tally(const FusedClassify& fc, const StageTally<NA>& tally) {
+  if (NA == 0 || fc.counts == nullptr) return;
+  __shared__ uint32_t sh[kMaxAlphas][3][kRankThreads / 32];
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+#pragma unroll
+  for (int a = 0; a < NA; ++a) {
+    uint32_t v1 = tally.c1[a], v3 = tally.c3[a], v2 = tally.seen - tally.c1[a] - tally.c3[a];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, o);
+      v2 += __shfl_xor_sync(0xFFFFFFFFu, v2, o);
+      v3 += __shfl_xor_sync(0xFFFFFFFFu, v3, o);
+    }
+    if (l == 0) { sh[a][0][w] = v1; sh[a][1][w] = v2; sh[a][2][w] = v3; }
+  }
+  __syncthreads();
+  if ((int)threadIdx.x < NA * 3) {
+    const int a = threadIdx.x / 3, i = threadIdx.x % 3;
+    uint32_t t = 0;
+    for (int q = 0; q < kRankThreads / 32; ++q) t += sh[a][i][q];
+    if (t) atomicAdd(fc.counts + threadIdx.x, t);
+  }
+}
+
 template <int NA>
 __global__ void __launch_bounds__(kRankThreads)
 rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restrict__ calib, int n,
             int ns, int P, int L, uint32_t* __restrict__ numer, float* __restrict__ pvalue,
             const FusedClassify fc) {
   extern __shared__ float sp[];
-  uint32_t c1[NA > 0 ? NA : 1] = {}, c3[NA > 0 ? NA : 1] = {}, seen = 0;
+  StageTally<NA> tally;
   const int slots = (1 << P) - 1;
   // With the whole buffer in the table (L == 0) the p-values of all n + 2 possible numerators are tabulated
   // behind it once per block (the same correctly rounded division), so a candidate costs one load, not a divide.
@@ -186,7 +253,7 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
       for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
     }
     rank_four(s, sp, P, L, calib, n, vec8, r);
-    float p[4];
+    float p[4] = {qnan, qnan, qnan, qnan};
     if (tabulated) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) p[e] = ptab[r[e]];
@@ -194,57 +261,165 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
 #pragma unroll
       for (int e = 0; e < 4; ++e) p[e] = r[e] ? __fdiv_rn((float)r[e], denom) : qnan;
     }
-    if (full) {
-      *reinterpret_cast<uint4*>(numer + j) = make_uint4(r[0], r[1], r[2], r[3]);
-      if (pvalue) *reinterpret_cast<float4*>(pvalue + j) = make_float4(p[0], p[1], p[2], p[3]);
-    } else {
-      for (int e = 0; e < 4 && j + e < Nc; ++e) {
-        numer[j + e] = r[e];
-        if (pvalue) pvalue[j + e] = p[e];
-      }
-    }
-    if (NA > 0) {
-      const int valid = full ? 4 : (int)(Nc - j);
-      seen += (uint32_t)valid;
-#pragma unroll
-      for (int a = 0; a < NA; ++a) {
-        uint32_t st[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          st[e] = stage_of(r[e], fc.k_alpha[a]);
-          c1[a] += (e < valid) && (st[e] == 1u);
-          c3[a] += (e < valid) && (st[e] == 3u);
-        }
-        if (full) {
-          *reinterpret_cast<uint32_t*>(fc.stage[a] + j) = st[0] | (st[1] << 8) | (st[2] << 16) | (st[3] << 24);
-        } else {
-          for (int e = 0; e < valid; ++e) fc.stage[a][j + e] = (uint8_t)st[e];
-        }
-      }
-    }
+    emit_four<NA>(j, Nc, full, r, p, numer, pvalue, fc, tally);
   }
-  if (NA > 0 && fc.counts != nullptr) {
-    __shared__ uint32_t sh[kMaxAlphas][3][kRankThreads / 32];
-    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+  flush_tally<NA>(fc, tally);
+}
+
+// ---------------------------------------------------------------------------------------------
+// K3, bucket form: many candidates against a buffer that fits in shared memory (n <= kBucketMaxN).
+//
+// A search tree costs a candidate log2(n) dependent shared-memory loads, which bounds the kernel by the
+// shared-memory pipe and by instruction issue long before HBM.  Here a candidate is first mapped to one of B
+// buckets of equal width in the monotone key space between the smallest and largest buffer entry
+// (bucket = ((key - key_lo) * mul) >> 32, clamped: a non-decreasing function of the key, applied alike to
+// candidates and buffer entries).  start[b] = number of buffer entries in buckets below b, so entries before
+// start[bucket(s)] are below s, entries from start[bucket(s) + 1] on are not, and only the entries of the
+// candidate's own bucket are compared with it.  With B >= 4n a bucket seldom holds more than one entry: the
+// candidate reads the two entries from start[b] on (entries beyond its bucket never compare below it, so no
+// count is needed); only in a bucket marked as holding more than two does it search the rest of the bucket.
+// Any distribution is handled exactly; a clustered one merely sends more candidates to that search.
+// ---------------------------------------------------------------------------------------------
+constexpr int kBucketMaxN = 8191;
+constexpr int kBucketMaxLog2 = 15;   // at most 32768 buckets (128 KB)
+constexpr int kBucketPad = 2;        // NaN entries behind the buffer copy, so probes need no bounds check
+constexpr int64_t kBucketMinCandidates = 1 << 16;
+
+struct BucketMap {
+  uint32_t key_lo, mul, last;  // last = B - 1
+};
+// value: canonical (no -0; one NaN pattern)
+__device__ __forceinline__ uint32_t bucket_of(float value, const BucketMap& m) {
+  const uint32_t u = __float_as_uint(value);
+  const uint32_t key = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
+  const uint32_t x = max(key, m.key_lo) - m.key_lo;
+  return min(__umulhi(x, m.mul), m.last);
+}
+
+template <int NA>
+__global__ void __launch_bounds__(kRankThreads, 1)
+rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restrict__ calib, int n, int Blog2,
+                   uint32_t* __restrict__ numer, float* __restrict__ pvalue, const FusedClassify fc) {
+  extern __shared__ uint32_t bsm[];
+  const int B = 1 << Blog2;
+  uint32_t* const start = bsm;                                         // [B + 1]
+  float* const buf = reinterpret_cast<float*>(bsm + B + 1);           // [n + kBucketPad]
+  float* const ptab = buf + n + kBucketPad;                            // [n + 2]
+  __shared__ BucketMap map_sh;
+  __shared__ uint32_t warp_max[kRankThreads / 32];
+  const float qnan = __uint_as_float(0x7FC00000u);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int t = threadIdx.x; t <= B; t += kRankThreads) start[t] = t == B ? (uint32_t)n : 0u;
+  for (int t = threadIdx.x; t < n + kBucketPad; t += kRankThreads)
+    buf[t] = t < n ? __uint_as_float(canonical_bits(__ldg(calib + t))) : qnan;
+  if (pvalue)
+    for (int t = threadIdx.x; t <= n + 1; t += kRankThreads)
+      ptab[t] = t ? __fdiv_rn((float)t, (float)(n + 1)) : qnan;
+  if (threadIdx.x == 0) {
+    const uint32_t lo = key_of_bits(canonical_bits(__ldg(calib)));
+    const uint32_t hi = key_of_bits(canonical_bits(__ldg(calib + n - 1)));
+    const unsigned long long range = hi >= lo ? (unsigned long long)(hi - lo) + 1ull : 1ull;
+    const unsigned long long mul = ((unsigned long long)B << 32) / range;
+    map_sh.key_lo = lo;
+    map_sh.mul = mul > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)mul;
+    map_sh.last = (uint32_t)(B - 1);
+  }
+  __syncthreads();
+  const BucketMap map = map_sh;
+  // start[b + 1] <- 1 + (largest index of an entry in bucket b); a running maximum then gives every start[b].
+  for (int t = threadIdx.x; t < n; t += kRankThreads) atomicMax(&start[bucket_of(buf[t], map) + 1u], (uint32_t)t + 1u);
+  __syncthreads();
+  {
+    // warp w owns start[w * seg .. (w + 1) * seg), seg = B / 32, read 32 consecutive words at a time
+    const int seg = B >> 5;
+    uint32_t* const mine = start + warp * seg;
+    uint32_t m = 0;
+    for (int i = lane; i < seg; i += 32) m = max(m, mine[i]);
 #pragma unroll
-    for (int a = 0; a < NA; ++a) {
-      uint32_t v1 = c1[a], v3 = c3[a], v2 = seen - c1[a] - c3[a];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, o);
-        v2 += __shfl_xor_sync(0xFFFFFFFFu, v2, o);
-        v3 += __shfl_xor_sync(0xFFFFFFFFu, v3, o);
-      }
-      if (l == 0) { sh[a][0][w] = v1; sh[a][1][w] = v2; sh[a][2][w] = v3; }
-    }
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (lane == 0) warp_max[warp] = m;
     __syncthreads();
-    if ((int)threadIdx.x < NA * 3) {
-      const int a = threadIdx.x / 3, i = threadIdx.x % 3;
-      uint32_t t = 0;
-      for (int q = 0; q < kRankThreads / 32; ++q) t += sh[a][i][q];
-      if (t) atomicAdd(fc.counts + threadIdx.x, t);
+    uint32_t carry = 0;
+    for (int w = 0; w < warp; ++w) carry = max(carry, warp_max[w]);
+    for (int i = 0; i < seg; i += 32) {
+      uint32_t v = (i + lane < seg) ? mine[i + lane] : 0u;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, v, o);
+        if (lane >= o) v = max(v, up);
+      }
+      v = max(v, carry);
+      if (i + lane < seg) mine[i + lane] = v;
+      carry = __shfl_sync(0xFFFFFFFFu, v, 31);
     }
   }
+  __syncthreads();
+  {
+    // mark the buckets that hold more than two entries (bit 31 of their start word)
+    uint32_t crowded = 0;
+    for (int i = 0, b = threadIdx.x; b < B; ++i, b += kRankThreads) crowded |= (start[b + 1] - start[b] > 2u ? 1u : 0u) << i;
+    __syncthreads();
+    for (int i = 0, b = threadIdx.x; b < B; ++i, b += kRankThreads)
+      if ((crowded >> i) & 1u) start[b] |= 0x80000000u;
+  }
+  __syncthreads();
+
+  StageTally<NA> tally;
+  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
+  const int64_t stride = (int64_t)gridDim.x * per_block;
+  int64_t j = (int64_t)blockIdx.x * per_block + (int64_t)threadIdx.x * kRankPerThread;
+  float4 nxt = make_float4(qnan, qnan, qnan, qnan);
+  if (j + 4 <= Nc) nxt = *reinterpret_cast<const float4*>(scores + j);
+  for (; j < Nc; j += stride) {
+    float s[4] = {nxt.x, nxt.y, nxt.z, nxt.w};
+    const bool full = j + kRankPerThread <= Nc;
+    if (!full) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
+    }
+    if (j + stride + 4 <= Nc) nxt = *reinterpret_cast<const float4*>(scores + j + stride);  // next round's scores
+    uint32_t word[4], below[4];
+    float p0[4], p1[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) word[e] = start[bucket_of(__fadd_rn(s[e], 0.f), map)];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const uint32_t st = word[e] & 0x7FFFFFFFu;
+      p0[e] = buf[st];
+      p1[e] = buf[st + 1];
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      below[e] = (word[e] & 0x7FFFFFFFu) + (p0[e] < s[e] ? 1u : 0u) + (p1[e] < s[e] ? 1u : 0u);
+    if ((word[0] | word[1] | word[2] | word[3]) & 0x80000000u) {
+      // a crowded bucket: if its first two entries are below the score, lower bound among the rest of the bucket
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if ((word[e] & 0x80000000u) && p1[e] < s[e]) {
+          int lo = (int)(word[e] & 0x7FFFFFFFu) + 2;
+          int len = (int)(start[bucket_of(__fadd_rn(s[e], 0.f), map) + 1u] & 0x7FFFFFFFu) - lo;
+          while (len > 0) {
+            const int half = len >> 1;
+            const bool less = buf[lo + half] < s[e];
+            lo = less ? lo + half + 1 : lo;
+            len = less ? len - half - 1 : half;
+          }
+          below[e] = (uint32_t)lo;
+        }
+      }
+    }
+    uint32_t r[4];
+    float p[4] = {qnan, qnan, qnan, qnan};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) r[e] = (s[e] != s[e]) ? 0u : (uint32_t)n - below[e] + 1u;  // NaN: no score
+    if (pvalue) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) p[e] = ptab[r[e]];
+    }
+    emit_four<NA>(j, Nc, full, r, p, numer, pvalue, fc, tally);
+  }
+  flush_tally<NA>(fc, tally);
 }
 
 // ---------------------------------------------------------------------------------------------

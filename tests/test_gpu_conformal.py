@@ -95,6 +95,38 @@ def test_rank_many_candidates_tied_clustered_and_special_data(n):
         assert np.array_equal(numer[idx], orc.conformal_numer_count(scores[idx], calib)), name
 
 
+@pytest.mark.parametrize("Nc,n", [(1 << 16, 1), ((1 << 16) + 3, 3), (1 << 18, 1000), (300007, 8191), (70001, 4096)])
+def test_rank_bucket_form_bit_exact(Nc, n):
+    """Many candidates against a small buffer take the bucket form of the rank kernel: smooth data (nearly every
+    bucket holds at most one entry), then data packed into a sliver of the key range beside far outliers (most
+    candidates search inside one bucket), with and without the p-value output and with fused thresholds."""
+    smooth = np.sort(inputs.lognormal_scores(40 + n, n))
+    packed = np.float32(1.0) + np.float32(1e-4) * inputs.lognormal_scores(41 + n, n)
+    if n >= 3:
+        packed[:2] = np.array([-3e38, 3e38], np.float32)
+    packed = np.sort(packed)
+    for calib, scores in ((smooth, inputs.lognormal_scores(42 + Nc, Nc)),
+                          (packed, np.float32(1.0) + np.float32(1e-4) * inputs.lognormal_scores(43 + Nc, Nc))):
+        scores[:6] = np.array([np.nan, -np.inf, np.inf, 0.0, -0.0, calib[n // 2]], np.float32)
+        numer = check_rank(scores, calib)
+        idx = np.concatenate([np.arange(6), np.arange(6, Nc, 2503)])
+        assert np.array_equal(numer[idx], orc.conformal_numer_count(scores[idx], calib))
+        numer_only, _ = gpu_rank(scores, calib, want_p=False)
+        assert np.array_equal(numer_only, numer)
+    Nf = Nc - Nc % 16
+    alphas = (0.05, 0.1, 0.2)
+    s, c = dev(scores[:Nf]), dev(calib)
+    out_numer, p = poison((Nf,), torch.int32), poison((Nf,), torch.float32)
+    stage, counts = poison((3, Nf), torch.uint8), poison((3, 3), torch.int32)
+    binding.rank_classify(s, c, n, alphas, out_numer, p, stage, counts)
+    torch.cuda.synchronize()
+    assert np.array_equal(host_u32(out_numer), numer[:Nf])
+    for a, alpha in enumerate(alphas):
+        want_stage, want_counts = orc.classify(numer[:Nf], n, alpha)
+        assert np.array_equal(stage[a].cpu().numpy(), want_stage)
+        assert np.array_equal(host_u32(counts[a]), want_counts)
+
+
 def test_rank_buffer_not_32_byte_aligned():
     # the kernel's 256-bit loads need a 32-byte aligned buffer; any other 4-byte aligned pointer takes the scalar path
     n, Nc = 100000, 1 << 17
