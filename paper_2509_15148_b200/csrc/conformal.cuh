@@ -276,9 +276,9 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
 // candidates and buffer entries).  start[b] = number of buffer entries in buckets below b, so entries before
 // start[bucket(s)] are below s, entries from start[bucket(s) + 1] on are not, and only the entries of the
 // candidate's own bucket are compared with it.  With B >= 4n a bucket seldom holds more than one entry: the
-// candidate reads the two entries from start[b] on (entries beyond its bucket never compare below it, so no
-// count is needed); only in a bucket marked as holding more than two does it search the rest of the bucket.
-// Any distribution is handled exactly; a clustered one merely sends more candidates to that search.
+// start word carries min(entries in the bucket, 3) in its top bits; a candidate reads nothing from an empty
+// bucket, one or two entries otherwise, and only in a bucket of three or more does it search the rest of the
+// bucket.  Any distribution is handled exactly; a clustered one merely sends more candidates to that search.
 // ---------------------------------------------------------------------------------------------
 constexpr int kBucketMaxN = 8191;
 constexpr int kBucketMaxLog2 = 15;   // at most 32768 buckets (128 KB)
@@ -288,7 +288,9 @@ constexpr int64_t kBucketMinCandidates = 1 << 16;
 struct BucketMap {
   uint32_t key_lo, mul, last;  // last = B - 1
 };
-// value: canonical (no -0; one NaN pattern)
+// Buffer entries are canonicalised first (no -0, one NaN pattern that has the largest key).  Candidates are not:
+// the key of -0 is the one just below that of +0, so a -0 candidate lands in the bucket of +0 or in the one
+// before it, and in both cases exactly the entries below zero precede its bucket's entries that are not.
 __device__ __forceinline__ uint32_t bucket_of(float value, const BucketMap& m) {
   const uint32_t u = __float_as_uint(value);
   const uint32_t key = u ^ ((uint32_t)((int32_t)u >> 31) | 0x80000000u);
@@ -356,12 +358,14 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
   }
   __syncthreads();
   {
-    // mark the buckets that hold more than two entries (bit 31 of their start word)
-    uint32_t crowded = 0;
-    for (int i = 0, b = threadIdx.x; b < B; ++i, b += kRankThreads) crowded |= (start[b + 1] - start[b] > 2u ? 1u : 0u) << i;
+    // bits 31:30 of a start word: min(entries in the bucket, 3)
+    uint64_t cls = 0;
+    for (int i = 0, b = threadIdx.x; b < B; ++i, b += kRankThreads) {
+      const uint32_t cnt = start[b + 1] - start[b];
+      cls |= (uint64_t)(cnt < 3u ? cnt : 3u) << (2 * i);
+    }
     __syncthreads();
-    for (int i = 0, b = threadIdx.x; b < B; ++i, b += kRankThreads)
-      if ((crowded >> i) & 1u) start[b] |= 0x80000000u;
+    for (int i = 0, b = threadIdx.x; b < B; ++i, b += kRankThreads) start[b] |= (uint32_t)((cls >> (2 * i)) & 3u) << 30;
   }
   __syncthreads();
 
@@ -380,25 +384,26 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
     }
     if (j + stride + 4 <= Nc) nxt = *reinterpret_cast<const float4*>(scores + j + stride);  // next round's scores
     uint32_t word[4], below[4];
-    float p0[4], p1[4];
+    float p0[4] = {qnan, qnan, qnan, qnan}, p1[4] = {qnan, qnan, qnan, qnan};
 #pragma unroll
-    for (int e = 0; e < 4; ++e) word[e] = start[bucket_of(__fadd_rn(s[e], 0.f), map)];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const uint32_t st = word[e] & 0x7FFFFFFFu;
-      p0[e] = buf[st];
-      p1[e] = buf[st + 1];
-    }
+    for (int e = 0; e < 4; ++e) word[e] = start[bucket_of(s[e], map)];
+    // Most buckets are empty: lanes whose bucket is read nothing, which also spares shared-memory bank conflicts.
 #pragma unroll
     for (int e = 0; e < 4; ++e)
-      below[e] = (word[e] & 0x7FFFFFFFu) + (p0[e] < s[e] ? 1u : 0u) + (p1[e] < s[e] ? 1u : 0u);
-    if ((word[0] | word[1] | word[2] | word[3]) & 0x80000000u) {
-      // a crowded bucket: if its first two entries are below the score, lower bound among the rest of the bucket
+      if (word[e] >= (1u << 30)) p0[e] = buf[word[e] & 0x3FFFFFFFu];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (word[e] >= (2u << 30)) p1[e] = buf[(word[e] & 0x3FFFFFFFu) + 1u];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      below[e] = (word[e] & 0x3FFFFFFFu) + (p0[e] < s[e] ? 1u : 0u) + (p1[e] < s[e] ? 1u : 0u);
+    if (max(max(word[0], word[1]), max(word[2], word[3])) >= (3u << 30)) {
+      // a bucket of three or more: if its first two entries are below the score, lower bound among the rest of it
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        if ((word[e] & 0x80000000u) && p1[e] < s[e]) {
-          int lo = (int)(word[e] & 0x7FFFFFFFu) + 2;
-          int len = (int)(start[bucket_of(__fadd_rn(s[e], 0.f), map) + 1u] & 0x7FFFFFFFu) - lo;
+        if (word[e] >= (3u << 30) && p1[e] < s[e]) {
+          int lo = (int)(word[e] & 0x3FFFFFFFu) + 2;
+          int len = (int)(start[bucket_of(s[e], map) + 1u] & 0x3FFFFFFFu) - lo;
           while (len > 0) {
             const int half = len >> 1;
             const bool less = buf[lo + half] < s[e];
