@@ -181,7 +181,9 @@ def conformal_stress(torch, binding, peaks):
     counts3 = torch.empty((len(cfg["alphas"]), 3), dtype=torch.int32, device=dev)
     ws = torch.empty(binding.calib_workspace_bytes(cap, k), dtype=torch.uint8, device=dev)
 
-    def sequence():
+    index = torch.empty(binding.calib_index_bytes(cap), dtype=torch.uint8, device=dev)
+
+    def sequence_plain():
         buf[:n0] = calib0
         n = n0
         for t in range(steps):
@@ -189,7 +191,18 @@ def conformal_stress(torch, binding, peaks):
             n = binding.calib_update(buf, n, news[t], ws)
         return n
 
+    def sequence():
+        # the calibration state is the buffer and its search index; every update rebuilds the index
+        buf[:n0] = calib0
+        binding.calib_index_build(buf, n0, index)
+        n = n0
+        for t in range(steps):
+            binding.rank_classify_indexed(scores, buf, n, index, cfg["alphas"], numer, p, stage3, counts3)
+            n = binding.calib_update_indexed(buf, n, news[t], index, ws)
+        return n
+
     graph_ms = make_graph_timer(torch)
+    ms_seq_plain = graph_ms(sequence_plain)
     ms_seq = graph_ms(sequence)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     eager = []
@@ -205,14 +218,19 @@ def conformal_stress(torch, binding, peaks):
     ms_cls = graph_ms(lambda: binding.classify(numer, n_end, 0.1, stage, counts), reps=20)
     ms_upd = graph_ms(lambda: binding.calib_update(buf, n_end, news[0], ws), reps=20)
     ms_fused = graph_ms(lambda: binding.rank_classify(scores, buf, n_end, cfg["alphas"], numer, p, stage3, counts3), reps=20)
+    binding.calib_index_build(buf, n_end, index)
+    ms_fused_ix = graph_ms(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, cfg["alphas"], numer, p, stage3,
+                                                                 counts3), reps=20)
+    ms_upd_ix = graph_ms(lambda: binding.calib_update_indexed(buf, n_end, news[0], index, ws), reps=20)
     rank_bytes = 12.0 * Nc + 4.0 * n_end
     cls_bytes = 5.0 * Nc
     fused_bytes = rank_bytes + len(cfg["alphas"]) * Nc
     out = {
         "workload": f"conformal-only stress: Nc={Nc}, n {n0}->{cap}, k={k}, {steps} steps, alphas {list(cfg['alphas'])}",
-        "step": "atts_rank_classify (3 alphas, one launch) + atts_calib_update",
+        "step": "atts_rank_classify_indexed (3 alphas, one launch) + atts_calib_update_indexed",
         "pvalues_per_s": Nc * steps / (ms_seq * 1e-3),
         "ms_sequence": ms_seq, "ms_sequence_eager_launches": min(eager),
+        "ms_sequence_without_index": ms_seq_plain, "pvalues_per_s_without_index": Nc * steps / (ms_seq_plain * 1e-3),
         "timing": "64-step sequence captured in one CUDA graph, events around the replay, best of 5; working set "
                   "(<= 14 MB) is L2-resident, so GB/s are algorithmic bytes over time, not DRAM traffic",
         "rank_us": ms_rank * 1e3, "rank_gbs": rank_bytes / (ms_rank * 1e-3) / 1e9,
@@ -220,6 +238,8 @@ def conformal_stress(torch, binding, peaks):
         "classify_us": ms_cls * 1e3, "classify_gbs": cls_bytes / (ms_cls * 1e-3) / 1e9,
         "update_us": ms_upd * 1e3,
         "rank_classify_fused_us": ms_fused * 1e3, "rank_classify_fused_gbs": fused_bytes / (ms_fused * 1e-3) / 1e9,
+        "rank_classify_indexed_us": ms_fused_ix * 1e3, "rank_classify_indexed_gbs": fused_bytes / (ms_fused_ix * 1e-3) / 1e9,
+        "update_indexed_us": ms_upd_ix * 1e3,
     }
     del scores, numer, p, stage, stage3
     out.update(conformal_scaled(torch, binding, peaks, graph_ms))

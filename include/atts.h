@@ -43,13 +43,15 @@ typedef enum {
   ATTS_ERR_ARCH = 7,      /* the current device is not sm_100                            */
   ATTS_ERR_CUDA = 8,      /* a CUDA runtime or driver call failed                        */
   ATTS_ERR_TIMEOUT = 9,   /* reported by atts_last_device_status: a bounded device wait expired */
-  ATTS_ERR_SCRATCH_LIMIT = 10 /* atts_calib_update_static: the sizes exceed its built-in scratch */
+  ATTS_ERR_SCRATCH_LIMIT = 10, /* atts_calib_update_static: the sizes exceed its built-in scratch */
+  ATTS_ERR_INDEX = 11     /* reported by atts_last_device_status: a calibration index did not match its buffer */
 } atts_status;
 
 /* Bits of the device status word returned by atts_last_device_status. */
 #define ATTS_DEV_TOKEN_ID_RANGE 1u /* a token id was outside [0, V): that row's log-prob is NaN */
 #define ATTS_DEV_WAIT_EXPIRED 2u   /* a pipeline wait in the scoring kernel ran out; outputs invalid */
 #define ATTS_DEV_GROUP_ID_RANGE 4u /* a group id was outside [0, G): that candidate has numer 0 */
+#define ATTS_DEV_INDEX_STALE 8u    /* atts_rank_classify_indexed: the index was built for another n; no output written */
 
 /* Stage labels written by atts_classify (the three stages of the rejection-sampling pipeline,
  * Sec. 3.3): the highest stage a sample reaches in this turn. */
@@ -253,6 +255,37 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
                       int64_t* n_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Calibration index (a convenience of this library for speed; the paper has no counterpart; results are
+ * those of Eq. p-value, byte for byte what atts_rank_classify writes).
+ *
+ * Ranking many candidates against a buffer too large for shared memory is bound by the divergent loads
+ * of each candidate's search.  A small index kept beside the buffer - the last entry of every aligned group
+ * of 8 entries, and the last entry of every group of 64 laid out as a search tree - lets a candidate finish
+ * with two 32-byte loads.  The index describes one fill n of one buffer: rebuild it whenever the buffer
+ * changes.  atts_calib_update_indexed does so in the pass that writes the merged buffer back, at no extra
+ * launch; atts_calib_index_build does it for a buffer filled some other way.
+ *
+ *   atts_calib_index_bytes   host out *bytes: size of an index for buffers of up to `cap` entries,
+ *                            0 <= cap <= 524,223 (else ATTS_ERR_SHAPE: use the calls without an index)
+ *   index         dev  256-byte aligned, at least atts_calib_index_bytes(n) bytes (ATTS_ERR_WORKSPACE)
+ *   calib_sorted  dev  as for atts_conformal_rank; atts_rank_classify_indexed also needs it 32-byte aligned
+ *   atts_calib_update_indexed   arguments and result as atts_calib_update; afterwards `index` describes
+ *                            calib[0, n + k)
+ *   atts_rank_classify_indexed  arguments and outputs as atts_rank_classify, but n_alpha may be 0 (rank and
+ *                            p-values only; stage and stage_counts are then ignored).  If `index` was built
+ *                            for another n nothing is written and ATTS_DEV_INDEX_STALE is recorded
+ *                            (atts_last_device_status then returns ATTS_ERR_INDEX).
+ */
+int atts_calib_index_bytes(int64_t cap, size_t* bytes);
+int atts_calib_index_build(const float* calib_sorted, int64_t n, void* index, size_t index_bytes, void* cuda_stream);
+int atts_calib_update_indexed(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k,
+                              int64_t* n_out, void* index, size_t index_bytes, void* workspace,
+                              size_t workspace_bytes, void* cuda_stream);
+int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
+                               const void* index, const double* alphas, int32_t n_alpha, uint32_t* numer,
+                               float* pvalue, uint8_t* stage, uint32_t* stage_counts, void* cuda_stream);
+
+/*
  * Allocation-free variant of atts_calib_update (a convenience of this library; the paper has no
  * counterpart).  Same result, bit for bit, but the caller passes no workspace: the scratch is a
  * fixed array inside the library's device image.
@@ -288,7 +321,8 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
 /*
  * Waits for `cuda_stream`, then returns in *bits (host out) the OR of the ATTS_DEV_* conditions
  * device code has recorded on the current device since the last call, and clears them.  Returns
- * ATTS_ERR_TIMEOUT if ATTS_DEV_WAIT_EXPIRED is among them, else ATTS_OK.
+ * ATTS_ERR_TIMEOUT if ATTS_DEV_WAIT_EXPIRED is among them, else ATTS_ERR_INDEX if ATTS_DEV_INDEX_STALE is,
+ * else ATTS_OK.
  */
 int atts_last_device_status(void* cuda_stream, uint32_t* bits);
 

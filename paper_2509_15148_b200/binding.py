@@ -20,10 +20,11 @@ EXPORTS = (
     "atts_calib_update_static", "atts_rank_classify", "atts_score_logprob_scaled", "atts_rms_inv",
     "atts_threshold", "atts_classify_threshold", "atts_conformal_rank_conditional", "atts_classify_conditional",
     "atts_debug_score_plan", "atts_debug_score_unit", "atts_score_slice", "atts_score_combine",
+    "atts_calib_index_bytes", "atts_calib_index_build", "atts_calib_update_indexed", "atts_rank_classify_indexed",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
-DEV_TOKEN_ID_RANGE, DEV_WAIT_EXPIRED, DEV_GROUP_ID_RANGE = 1, 2, 4
+DEV_TOKEN_ID_RANGE, DEV_WAIT_EXPIRED, DEV_GROUP_ID_RANGE, DEV_INDEX_STALE = 1, 2, 4, 8
 
 _lib = None
 
@@ -78,6 +79,12 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
                                       c_size_t, c_void_p]
     lib.atts_last_device_status.argtypes = [c_void_p, POINTER(c_uint32)]
     lib.atts_calib_update_static.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p]
+    lib.atts_calib_index_bytes.argtypes = [c_int64, POINTER(c_size_t)]
+    lib.atts_calib_index_build.argtypes = [c_void_p, c_int64, c_void_p, c_size_t, c_void_p]
+    lib.atts_calib_update_indexed.argtypes = [c_void_p, c_int64, c_int64, c_void_p, c_int64, POINTER(c_int64), c_void_p,
+                                              c_size_t, c_void_p, c_size_t, c_void_p]
+    lib.atts_rank_classify_indexed.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, POINTER(c_double), c_int32,
+                                               c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.atts_profile_begin.argtypes = [c_int]
     lib.atts_profile_end.argtypes = [POINTER(ctypes.c_float), c_int, POINTER(c_int)]
     for name in EXPORTS[2:]:
@@ -221,6 +228,41 @@ def calib_update(calib, n: int, new_scores, workspace) -> int:
     return n_out.value
 
 
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def calib_index_bytes(cap: int) -> int:
+    out = c_size_t(0)
+    _check(load().atts_calib_index_bytes(cap, ctypes.byref(out)), "atts_calib_index_bytes")
+    return out.value
+
+
+def calib_index_build(calib_sorted, n: int, index) -> None:
+    """Write into `index` (uint8 tensor) the search index of the first n entries of calib_sorted."""
+    _check(load().atts_calib_index_build(_ptr(calib_sorted), n, _ptr(index), _nbytes(index), _stream()),
+           "atts_calib_index_build")
+
+
+def calib_update_indexed(calib, n: int, new_scores, index, workspace) -> int:
+    """:func:`calib_update` that also leaves in `index` the search index of the updated buffer. Returns n + k."""
+    n_out = c_int64(0)
+    k = 0 if new_scores is None else new_scores.numel()
+    _check(load().atts_calib_update_indexed(_ptr(calib), n, calib.numel(), _ptr(new_scores), k, ctypes.byref(n_out),
+                                            _ptr(index), _nbytes(index), _ptr(workspace), _nbytes(workspace), _stream()),
+           "atts_calib_update_indexed")
+    return n_out.value
+
+
+def rank_classify_indexed(scores, calib_sorted, n: int, index, alphas, numer, pvalue=None, stage=None,
+                          stage_counts=None) -> None:
+    """:func:`rank_classify` with the buffer's search index; alphas may be empty (ranks and p-values only)."""
+    arr = (c_double * max(len(alphas), 1))(*[float(a) for a in alphas])
+    _check(load().atts_rank_classify_indexed(_ptr(scores), scores.numel(), _ptr(calib_sorted), n, _ptr(index), arr,
+                                             len(alphas), _ptr(numer), _ptr(pvalue), _ptr(stage), _ptr(stage_counts),
+                                             _stream()), "atts_rank_classify_indexed")
+
+
 STATIC_MAX_TOTAL, STATIC_MAX_NEW = 65536, 16384
 
 
@@ -238,12 +280,11 @@ def calib_update_static(calib, n: int, new_scores) -> int:
 
 
 def last_device_status() -> int:
-    """Synchronises the current stream; returns and clears the device status bits. Raises on an expired wait."""
+    """Synchronises the current stream; returns and clears the device status bits. Raises on an expired wait or a
+    stale calibration index."""
     bits = c_uint32(0)
     st = load().atts_last_device_status(_stream(), ctypes.byref(bits))
-    if st not in (0, 9):
-        raise AttsError(st, "atts_last_device_status")
-    if st == 9:
+    if st != 0:
         raise AttsError(st, "atts_last_device_status")
     return bits.value
 

@@ -81,6 +81,11 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaFuncSetAttribute(rank_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       const int bucket_smem = 4 * ((1 << kBucketMaxLog2) + 1 + 2 * kBucketMaxN + kBucketPad + 2);
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
@@ -210,6 +215,7 @@ const char* atts_strerror(int status) {
     case ATTS_ERR_TIMEOUT: return "a bounded wait on the device expired";
     case ATTS_ERR_SCRATCH_LIMIT:
       return "sizes exceed the built-in scratch of the allocation-free entry point (n + k <= 65536, k <= 16384)";
+    case ATTS_ERR_INDEX: return "the calibration index was built for another fill of the buffer";
     default: return "unknown status";
   }
 }
@@ -566,6 +572,34 @@ int atts_classify_conditional(const uint32_t* numer, const uint32_t* denom, int6
   return launch_status();
 }
 
+// ---- calibration index (see rank_indexed_kernel) ----
+static inline int index_levels(int64_t n, int* ns_out) {
+  const int ns = (int)(n / 64) + 1;
+  int P = 1;
+  while ((1 << P) - 1 < ns) ++P;
+  *ns_out = ns;
+  return P;
+}
+static inline size_t index_bytes_for(int64_t n) {
+  return 4 * ((size_t)kIndexHeaderWords + kIndexTreeWords + 8 * ((size_t)(n / 64) + 1));
+}
+
+// Launches the index build for src[0, n); copy_to != nullptr: also copies src to copy_to.
+static int launch_index_build(const DeviceInfo* di, const float* src, float* copy_to, int64_t n, void* index,
+                              cudaStream_t stream) {
+  int ns = 0;
+  const int P = index_levels(n, &ns);
+  int64_t work = n > (1ll << P) ? n : (1ll << P);
+  if (work < 8 * (int64_t)ns) work = 8 * (int64_t)ns;
+  int64_t blocks = (work + 255) / 256;
+  if (blocks > (int64_t)di->sm_count * 8) blocks = (int64_t)di->sm_count * 8;
+  if (copy_to)
+    index_build_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(src, copy_to, (int)n, P, ns, static_cast<uint32_t*>(index));
+  else
+    index_build_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(src, nullptr, (int)n, P, ns, static_cast<uint32_t*>(index));
+  return launch_status();
+}
+
 // Workspace of atts_calib_update: [sorted new keys: min(k, kSortMaxK) u32][merged copy: n + k f32]
 int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes) {
   if (!bytes) return ATTS_ERR_NULL;
@@ -575,8 +609,8 @@ int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes) {
   return ATTS_OK;
 }
 
-int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
-                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static int calib_update_impl(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
+                             void* workspace, size_t workspace_bytes, void* cuda_stream, void* index, size_t index_bytes) {
   if (n < 0 || k < 0 || cap < 0 || cap >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
   if (n + k > cap) return ATTS_ERR_CAPACITY;
   if ((cap > 0 && !calib) || (k > 0 && (!new_scores || !workspace))) return ATTS_ERR_NULL;
@@ -587,9 +621,14 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
   const DeviceInfo* di;
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
+  if (index) {
+    if (n + k > kIndexMaxN) return ATTS_ERR_SHAPE;
+    if (!aligned(index, 256)) return ATTS_ERR_ALIGN;
+    if (index_bytes < index_bytes_for(n + k)) return ATTS_ERR_WORKSPACE;
+  }
   if (n_out) *n_out = n + k;
-  if (k == 0) return ATTS_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (k == 0) return index ? launch_index_build(di, calib, nullptr, n, index, stream) : ATTS_OK;
   const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
   uint32_t* sorted_keys = static_cast<uint32_t*>(workspace);
   float* merged = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up((size_t)kk * 4, 256));
@@ -598,7 +637,8 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
     int k2 = 1;
     while (k2 < k) k2 <<= 1;
     small_update_kernel<<<1, kSmallUpdThreads, (size_t)4 * (k2 + n), stream>>>(calib, (int)n, new_scores, (int)k, k2);
-    return launch_status();
+    if ((st = launch_status()) != ATTS_OK) return st;
+    return index ? launch_index_build(di, calib, nullptr, n + k, index, stream) : ATTS_OK;
   }
   // Sort the new keys, merge into the workspace, copy back.  Batches larger than one sort launch handles are
   // inserted slice by slice.
@@ -614,13 +654,28 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
     if (merge_blocks > di->sm_count * 4) merge_blocks = di->sm_count * 4;
     merge_kernel<<<merge_blocks, kMergeThreads, (size_t)kc * 4, stream>>>(calib, (int)cur, sorted_keys, kc, merged);
     if ((st = launch_status()) != ATTS_OK) return st;
-    if (cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+    if (index && off + kSortMaxK >= k) {
+      // last slice: the copy back also writes the index of the merged buffer
+      if ((st = launch_index_build(di, merged, calib, total, index, stream)) != ATTS_OK) return st;
+    } else if (cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
       cudaGetLastError();
       return ATTS_ERR_CUDA;
     }
     cur = total;
   }
   return ATTS_OK;
+}
+
+int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  return calib_update_impl(calib, n, cap, new_scores, k, n_out, workspace, workspace_bytes, cuda_stream, nullptr, 0);
+}
+
+int atts_calib_update_indexed(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
+                              void* index, size_t index_bytes, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+  if (!index) return ATTS_ERR_NULL;
+  return calib_update_impl(calib, n, cap, new_scores, k, n_out, workspace, workspace_bytes, cuda_stream, index, index_bytes);
 }
 
 int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
@@ -657,6 +712,74 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
   return ATTS_OK;
 }
 
+int atts_calib_index_bytes(int64_t cap, size_t* bytes) {
+  if (!bytes) return ATTS_ERR_NULL;
+  if (cap < 0 || cap > kIndexMaxN) return ATTS_ERR_SHAPE;
+  *bytes = round_up(index_bytes_for(cap), 256);
+  return ATTS_OK;
+}
+
+int atts_calib_index_build(const float* calib_sorted, int64_t n, void* index, size_t index_bytes, void* cuda_stream) {
+  if (n < 0 || n > kIndexMaxN) return ATTS_ERR_SHAPE;
+  if (!index || (n > 0 && !calib_sorted)) return ATTS_ERR_NULL;
+  if (!aligned(calib_sorted, 4) || !aligned(index, 256)) return ATTS_ERR_ALIGN;
+  if (index_bytes < index_bytes_for(n)) return ATTS_ERR_WORKSPACE;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  return launch_index_build(di, calib_sorted, nullptr, n, index, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n, const void* index,
+                               const double* alphas, int32_t n_alpha, uint32_t* numer, float* pvalue, uint8_t* stage,
+                               uint32_t* stage_counts, void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n > kIndexMaxN) return ATTS_ERR_SHAPE;
+  if (n_alpha < 0 || n_alpha > kMaxAlphas) return ATTS_ERR_ARG;
+  if (n_alpha > 0 && !alphas) return ATTS_ERR_NULL;
+  for (int a = 0; a < n_alpha; ++a)
+    if (!(alphas[a] > 0.0 && alphas[a] < 1.0)) return ATTS_ERR_ARG;
+  if (!index || (Nc > 0 && (!scores || !numer || (n_alpha > 0 && !stage)))) return ATTS_ERR_NULL;
+  if (n > 0 && !calib_sorted) return ATTS_ERR_NULL;
+  if (!aligned(scores, 16) || !aligned(numer, 16) || !aligned(pvalue, 16) || !aligned(calib_sorted, 32) ||
+      !aligned(index, 256) || !aligned(stage, 16) || !aligned(stage_counts, 4) || (n_alpha > 1 && Nc % 16 != 0))
+    return ATTS_ERR_ALIGN;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (n_alpha > 0 && stage_counts &&
+      cudaMemsetAsync(stage_counts, 0, (size_t)n_alpha * 3 * sizeof(uint32_t), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  if (Nc == 0) return ATTS_OK;
+  FusedClassify fc{};
+  for (int a = 0; a < n_alpha; ++a) {
+    fc.k_alpha[a] = (uint32_t)floor(alphas[a] * (double)(n + 1));
+    fc.stage[a] = stage + (size_t)a * Nc;
+  }
+  fc.counts = n_alpha > 0 ? stage_counts : nullptr;
+  // A buffer that fits in shared memory, or few candidates, gain nothing from the index.
+  if (n <= kBucketMaxN || Nc < kIndexMinCandidates)
+    return launch_rank(di, scores, Nc, calib_sorted, n, numer, pvalue, n_alpha, fc, stream);
+  int ns = 0;
+  const int P = index_levels(n, &ns);
+  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
+  int64_t blocks = (Nc + per_block - 1) / per_block;
+  if (blocks > di->sm_count) blocks = di->sm_count;
+  const dim3 grid((unsigned)blocks), block(kRankThreads);
+  const size_t smem = (size_t)4 << P;
+  const uint32_t* ix = static_cast<const uint32_t*>(index);
+  switch (n_alpha) {
+    case 0: rank_indexed_kernel<0><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
+    case 1: rank_indexed_kernel<1><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
+    case 2: rank_indexed_kernel<2><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
+    case 3: rank_indexed_kernel<3><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
+    default: rank_indexed_kernel<4><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
+  }
+  return launch_status();
+}
+
 int atts_last_device_status(void* cuda_stream, uint32_t* bits) {
   if (!bits) return ATTS_ERR_NULL;
   const DeviceInfo* di;
@@ -671,7 +794,7 @@ int atts_last_device_status(void* cuda_stream, uint32_t* bits) {
     return ATTS_ERR_CUDA;
   }
   *bits = v;
-  return (v & ATTS_DEV_WAIT_EXPIRED) ? ATTS_ERR_TIMEOUT : ATTS_OK;
+  return (v & ATTS_DEV_WAIT_EXPIRED) ? ATTS_ERR_TIMEOUT : (v & ATTS_DEV_INDEX_STALE) ? ATTS_ERR_INDEX : ATTS_OK;
 }
 
 int atts_debug_score_plan(int64_t M, int64_t d, int64_t V, int32_t workers, int32_t ctas, int32_t* out) {

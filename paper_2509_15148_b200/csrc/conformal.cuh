@@ -428,6 +428,154 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
 }
 
 // ---------------------------------------------------------------------------------------------
+// K3, indexed form: many candidates against a buffer too large for shared memory.
+//
+// The plain kernel pays, per block, one strided load for each of up to 8191 splitters, and per candidate up to
+// three dependent 4-byte loads plus one 32-byte load from the L2-resident buffer; divergent loads are served at
+// one per cycle per SM, so they are what bounds it.  An index kept beside the buffer (rebuilt whenever the
+// buffer changes, in the pass that writes the buffer anyway) removes most of them:
+//   aux[i]  = calib[8 i + 7], the last entry of every aligned group of 8 (NaN where that lies beyond n);
+//   tree    = the entries aux[8 r + 7] = calib[64 r + 63], r < ns = n / 64 + 1 (the last one always NaN), as an
+//             implicit search tree in breadth-first order, ready to be copied into shared memory row by row.
+// A candidate descends the tree (P shared-memory steps) to its group of 64, reads that group's 8 aux entries
+// in one 32-byte load to find its group of 8, and reads that group in a second 32-byte load.
+// Layout of the index (32-bit words): [0] n  [1] P  [2] ns  [3..7] 0  [8 ..) tree, kIndexTreeWords  [..) aux, 8 ns.
+// ---------------------------------------------------------------------------------------------
+constexpr int kIndexHeaderWords = 8;
+constexpr int kIndexTreeWords = 1 << kRankMaxTableLog2;               // 8191 nodes + 1 pad
+constexpr int64_t kIndexMaxN = 64ll * ((1 << kRankMaxTableLog2) - 1) - 1;   // ns = n / 64 + 1 <= 8191
+constexpr int64_t kIndexMinCandidates = 1 << 14;
+
+// Slot, in the breadth-first table of a P-level tree, of the splitter with sorted rank r (inverse of the fill rule
+// of rank_kernel: node b at depth l holds rank (2q + 1) * 2^(P-1-l) - 1, q = b - 2^l).
+__device__ __forceinline__ int index_slot_of_rank(int r, int P) {
+  const int x = r + 1;
+  const int tz = __ffs(x) - 1;
+  const int depth = P - 1 - tz;
+  return (1 << depth) + (x >> (tz + 1)) - 1;
+}
+
+// Writes the index of src[0, n); with COPY also dst[e] = src[e] (the copy-back of a merge), so a calibration
+// update rebuilds the index in the pass that moves the merged buffer anyway.
+template <bool COPY>
+__global__ void __launch_bounds__(256)
+index_build_kernel(const float* __restrict__ src, float* __restrict__ dst, int n, int P, int ns,
+                   uint32_t* __restrict__ index) {
+  float* const tree = reinterpret_cast<float*>(index + kIndexHeaderWords);
+  float* const aux = tree + kIndexTreeWords;
+  const float qnan = __uint_as_float(0x7FC00000u);
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x;
+  if (tid < kIndexHeaderWords) index[tid] = tid == 0 ? (uint32_t)n : tid == 1 ? (uint32_t)P : tid == 2 ? (uint32_t)ns : 0u;
+  for (int e = tid; e < n; e += nthreads) {
+    const float v = src[e];
+    if (COPY) dst[e] = v;
+    if ((e & 7) == 7) aux[e >> 3] = v;
+    if ((e & 63) == 63) tree[index_slot_of_rank(e >> 6, P)] = v;
+  }
+  for (int i = (n >> 3) + tid; i < 8 * ns; i += nthreads) aux[i] = qnan;             // groups of 8 that end beyond n
+  for (int r = (n >> 6) + tid; r < (1 << P) - 1; r += nthreads) tree[index_slot_of_rank(r, P)] = qnan;
+}
+
+template <int P>
+__device__ __forceinline__ void rank_four_indexed(const float (&s)[4], const float* __restrict__ sp,
+                                                  const float* __restrict__ aux, const float* __restrict__ calib, int n,
+                                                  uint32_t (&numer)[4]) {
+  int g[4];
+  tree_descend<P>(s, sp, g);   // number of groups of 64 that lie entirely below the score
+  float w[4][8];
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(w[e][0]), "=f"(w[e][1]), "=f"(w[e][2]), "=f"(w[e][3]), "=f"(w[e][4]), "=f"(w[e][5]), "=f"(w[e][6]), "=f"(w[e][7])
+                 : "l"(aux + 8 * g[e]));
+  int h[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    int c = 0;
+#pragma unroll
+    for (int i = 0; i < 7; ++i) c += (w[e][i] < s[e]) ? 1 : 0;   // the eighth is the group's splitter: not below
+    h[e] = 8 * g[e] + c;                                         // groups of 8 that lie entirely below the score
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    // the last group may be cut short by n: its 32 bytes are still inside the 32-byte aligned span only if whole
+    if (8 * h[e] + 8 <= n) {
+      asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=f"(w[e][0]), "=f"(w[e][1]), "=f"(w[e][2]), "=f"(w[e][3]), "=f"(w[e][4]), "=f"(w[e][5]), "=f"(w[e][6]), "=f"(w[e][7])
+                   : "l"(calib + 8 * h[e]));
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) w[e][i] = (8 * h[e] + i < n) ? __ldg(calib + 8 * h[e] + i) : __uint_as_float(0x7FC00000u);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    int c = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) c += (w[e][i] < s[e]) ? 1 : 0;
+    const int below = 8 * h[e] + c;
+    numer[e] = (s[e] != s[e]) ? 0u : (uint32_t)(n - below) + 1u;   // NaN: no score
+  }
+}
+
+template <int NA>
+__global__ void __launch_bounds__(kRankThreads)
+rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restrict__ calib, int n, int P,
+                    const uint32_t* __restrict__ index, uint32_t* __restrict__ numer, float* __restrict__ pvalue,
+                    const FusedClassify fc, unsigned int* __restrict__ dev_status) {
+  extern __shared__ float sp[];
+  // an index built for another fill of the buffer would give wrong ranks silently: refuse it
+  if (__ldg(index) != (uint32_t)n || __ldg(index + 1) != (uint32_t)P) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(dev_status, 8u);
+    return;
+  }
+  const float* const tree = reinterpret_cast<const float*>(index + kIndexHeaderWords);
+  const float* const aux = tree + kIndexTreeWords;
+  for (int t = threadIdx.x; t < (1 << P) - 1; t += kRankThreads) sp[t] = __ldg(tree + t);
+  __syncthreads();
+  StageTally<NA> tally;
+  const float denom = (float)(n + 1);
+  const float qnan = __uint_as_float(0x7FC00000u);
+  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
+  for (int64_t base = (int64_t)blockIdx.x * per_block; base < Nc; base += (int64_t)gridDim.x * per_block) {
+    const int64_t j = base + (int64_t)threadIdx.x * kRankPerThread;
+    if (j >= Nc) continue;
+    float s[4];
+    uint32_t r[4];
+    const bool full = j + kRankPerThread <= Nc;
+    if (full) {
+      const float4 s4 = *reinterpret_cast<const float4*>(scores + j);
+      s[0] = s4.x; s[1] = s4.y; s[2] = s4.z; s[3] = s4.w;
+    } else {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
+    }
+    switch (P) {
+      case 1: rank_four_indexed<1>(s, sp, aux, calib, n, r); break;
+      case 2: rank_four_indexed<2>(s, sp, aux, calib, n, r); break;
+      case 3: rank_four_indexed<3>(s, sp, aux, calib, n, r); break;
+      case 4: rank_four_indexed<4>(s, sp, aux, calib, n, r); break;
+      case 5: rank_four_indexed<5>(s, sp, aux, calib, n, r); break;
+      case 6: rank_four_indexed<6>(s, sp, aux, calib, n, r); break;
+      case 7: rank_four_indexed<7>(s, sp, aux, calib, n, r); break;
+      case 8: rank_four_indexed<8>(s, sp, aux, calib, n, r); break;
+      case 9: rank_four_indexed<9>(s, sp, aux, calib, n, r); break;
+      case 10: rank_four_indexed<10>(s, sp, aux, calib, n, r); break;
+      case 11: rank_four_indexed<11>(s, sp, aux, calib, n, r); break;
+      case 12: rank_four_indexed<12>(s, sp, aux, calib, n, r); break;
+      default: rank_four_indexed<13>(s, sp, aux, calib, n, r); break;
+    }
+    float p[4] = {qnan, qnan, qnan, qnan};
+    if (pvalue) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) p[e] = r[e] ? __fdiv_rn((float)r[e], denom) : qnan;
+    }
+    emit_four<NA>(j, Nc, full, r, p, numer, pvalue, fc, tally);
+  }
+  flush_tally<NA>(fc, tally);
+}
+
+// ---------------------------------------------------------------------------------------------
 // K4  threshold + ordinal stage (accept iff p > alpha  <=>  numer > k_alpha).
 // ---------------------------------------------------------------------------------------------
 constexpr int kClassifyThreads = 256;

@@ -28,11 +28,11 @@ def test_header_symbols_are_exported():
 def test_strerror_and_version():
     assert binding.version() >= 100
     seen = set()
-    for code in range(0, 11):
+    for code in range(0, 12):
         s = binding.strerror(code)
         assert s and s != "unknown status"
         seen.add(s)
-    assert len(seen) == 11
+    assert len(seen) == 12
     assert binding.strerror(1234) == "unknown status"
 
 
@@ -60,6 +60,14 @@ def test_argument_errors_need_no_device():
     assert lib.atts_score_logprob(None, None, None, None, 8, 64, 100, 1, 7, None, None, None, 0, None) == 6
     assert lib.atts_score_logprob(None, None, None, None, 8, 64, 100, 1, 0, None, None, None, 0, None) == 1
     assert lib.atts_last_device_status(None, None) == 1
+    assert lib.atts_calib_index_bytes(524223, ctypes.byref(sz)) == 0 and sz.value % 256 == 0 and sz.value >= 4 * (8192 + 8 * 8191)
+    assert lib.atts_calib_index_bytes(524224, ctypes.byref(sz)) == 2                        # too large for an index
+    assert lib.atts_calib_index_bytes(10, None) == 1
+    assert lib.atts_calib_index_build(None, 10, None, 0, None) == 1
+    assert lib.atts_calib_index_build(None, 1 << 20, None, 0, None) == 2
+    assert lib.atts_calib_update_indexed(None, 10, 20, None, 5, None, None, 0, None, 0, None) == 1
+    assert lib.atts_rank_classify_indexed(None, 4, None, 0, None, None, 5, None, None, None, None, None) == 6
+    assert lib.atts_rank_classify_indexed(None, 4, None, 1 << 20, None, None, 0, None, None, None, None, None) == 2
 
 
 def test_no_device_means_error_not_fallback():

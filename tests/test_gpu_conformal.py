@@ -328,3 +328,95 @@ def test_randomised_sizes_and_value_mixes():
         buf, n2 = gpu_update(calib, new, n + k + 2)
         assert n2 == n + k
         assert np.array_equal(f32_bits(buf[:n2]), f32_bits(orc.calib_update(calib, new))), (case, n, k)
+
+
+def _index_for(calib_dev, n, cap=None):
+    ix = workspace(binding.calib_index_bytes(cap if cap is not None else n))
+    binding.calib_index_build(calib_dev, n, ix)
+    return ix
+
+
+@pytest.mark.parametrize("Nc,n", [(1 << 17, 8192), (100003, 8255), (1 << 16, 65536), (70001, 65543), (1 << 18, 327680),
+                                   (16384, 524223), (20000, 100), (100, 70000), (0, 9000)])
+def test_indexed_rank_equals_definition_and_plain_call(Nc, n):
+    """The indexed rank gives the numerators and p-value bits of the definition, on smooth data, on heavily tied data
+    and with special values at both ends of the buffer, with and without fused thresholds."""
+    for variant in ("smooth", "ties", "special"):
+        raw = inputs.lognormal_scores(900 + n, n)
+        scores = inputs.lognormal_scores(901 + Nc, Nc)
+        if variant == "ties":
+            raw, scores = np.round(raw, 1), np.round(scores, 1)
+        if variant == "special":
+            raw[:6] = np.array([-np.inf, -0.0, 0.0, np.inf, np.nan, np.nan], np.float32)
+        if Nc >= 8:
+            scores[:8] = np.array([np.nan, -np.inf, np.inf, 0.0, -0.0, raw[n // 2], 1e30, -1e30], np.float32)
+        calib = orc.calib_update(np.zeros(0, np.float32), raw)
+        c, s = dev(calib), dev(scores)
+        ix = _index_for(c, n)
+        numer, p = poison((Nc,), torch.int32), poison((Nc,), torch.float32)
+        binding.rank_classify_indexed(s, c, n, ix, (), numer, p)
+        torch.cuda.synchronize()
+        want = orc.conformal_numer_sorted(scores, calib)
+        assert np.array_equal(host_u32(numer), want), variant
+        assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want, n))), variant
+        if Nc:
+            idx = np.arange(0, Nc, max(Nc // 50, 1))
+            assert np.array_equal(want[idx], orc.conformal_numer_count(scores[idx], calib)), variant
+    Nf = Nc - Nc % 16
+    if Nf:
+        alphas = (0.05, 0.1, 0.2)
+        numer2, stage, counts = poison((Nf,), torch.int32), poison((3, Nf), torch.uint8), poison((3, 3), torch.int32)
+        binding.rank_classify_indexed(s[:Nf], c, n, ix, alphas, numer2, None, stage, counts)
+        torch.cuda.synchronize()
+        assert np.array_equal(host_u32(numer2), want[:Nf])
+        for a, alpha in enumerate(alphas):
+            ws, wc = orc.classify(want[:Nf], n, alpha)
+            assert np.array_equal(stage[a].cpu().numpy(), ws) and np.array_equal(host_u32(counts[a]), wc)
+    assert binding.last_device_status() == 0
+
+
+def test_indexed_update_sequence_keeps_buffer_and_index_in_step():
+    """A growing buffer: every update through the indexed entry point leaves the oracle's buffer and an index with
+    which the next rank is exact (small in-place path, general path, a slice-by-slice insert, an empty insert)."""
+    Nc = 1 << 16
+    scores = inputs.lognormal_scores(77, Nc)
+    s = dev(scores)
+    calib = np.sort(inputs.lognormal_scores(78, 5000))
+    cap = 5000 + 64 + 4096 + 40000 + 0 + 3000 + 8
+    buf = poison((cap,), torch.float32)
+    buf[:calib.size] = dev(calib)
+    ix = _index_for(buf, calib.size, cap)
+    n = calib.size
+    for step, k in enumerate((64, 4096, 40000, 0, 3000)):
+        new = inputs.lognormal_scores(80 + step, k)
+        ws = workspace(binding.calib_workspace_bytes(n, k))
+        n2 = binding.calib_update_indexed(buf, n, dev(new) if k else None, ix, ws)
+        calib = orc.calib_update(calib, new)
+        assert n2 == calib.size
+        n = n2
+        numer = poison((Nc,), torch.int32)
+        binding.rank_classify_indexed(s, buf, n, ix, (), numer)
+        torch.cuda.synchronize()
+        assert np.array_equal(f32_bits(buf[:n]), f32_bits(calib)), step
+        assert np.array_equal(host_u32(numer), orc.conformal_numer_sorted(scores, calib)), step
+    assert binding.last_device_status() == 0
+
+
+def test_stale_index_is_refused_and_argument_errors():
+    n, Nc = 20000, 1 << 15
+    calib = np.sort(inputs.lognormal_scores(90, n + 64))
+    c, s = dev(calib), dev(inputs.lognormal_scores(91, Nc))
+    ix = _index_for(c, n, n + 64)
+    numer = poison((Nc,), torch.int32)
+    binding.rank_classify_indexed(s, c, n + 64, ix, (), numer)           # index describes n, not n + 64
+    with pytest.raises(binding.AttsError) as err:
+        binding.last_device_status()
+    assert err.value.status == 11
+    assert np.all(host_u32(numer) == 0xFFFFFFFF)                         # nothing was written
+    assert binding.last_device_status() == 0                             # the bit was cleared
+    with pytest.raises(binding.AttsError) as err:                        # buffer not 32-byte aligned
+        binding.rank_classify_indexed(s, c[1:], n, ix, (), numer)
+    assert err.value.status == 3
+    with pytest.raises(binding.AttsError) as err:                        # index too small for this n
+        binding.calib_index_build(c, n + 64, ix[:1024])
+    assert err.value.status == 4
