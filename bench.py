@@ -119,6 +119,24 @@ def oracle_step(orc, Hb, Wb, ids, rows, N, calib, alpha):
     return orc.calib_update(calib, sc[~np.isnan(sc)])
 
 
+def oracle_conformal_steps(orc, steps_timed=16):
+    """The oracle on the first steps of the conformal-only workload: rank, p-values, three thresholds, insert."""
+    cfg = inputs.CONFORMAL_STRESS
+    scores = inputs.lognormal_scores(inputs.BASE_SEED + 1, cfg["Nc"])
+    calib = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, cfg["n0"]))
+    news = [inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, cfg["k"]) for t in range(steps_timed)]
+    t0 = time.perf_counter()
+    for t in range(steps_timed):
+        numer = orc.conformal_numer_sorted(scores, calib)
+        orc.pvalue(numer, calib.size)
+        for alpha in cfg["alphas"]:
+            orc.classify(numer, calib.size, alpha)
+        calib = orc.calib_update(calib, news[t])
+    dt = time.perf_counter() - t0
+    return {"value": cfg["Nc"] * steps_timed / dt, "unit": "p-values/s", "cores": 1, "kind": "oracle",
+            "sample": f"first {steps_timed} of {cfg['steps']} steps of the conformal-only workload in {dt:.1f} s"}
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -222,6 +240,32 @@ def conformal_stress(torch, binding, peaks):
     ms_fused_ix = graph_ms(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, cfg["alphas"], numer, p, stage3,
                                                                  counts3), reps=20)
     ms_upd_ix = graph_ms(lambda: binding.calib_update_indexed(buf, n_end, news[0], index, ws), reps=20)
+    # The same calls with a cold L2: 512 MB are written between repetitions, one call is timed by events (the events'
+    # own few microseconds are inside), median of 9.
+    scrub = torch.empty(128 << 20, dtype=torch.float32, device=dev)
+
+    def cold_us(fn):
+        ts = []
+        for _ in range(9):
+            scrub.fill_(1.0)
+            torch.cuda.synchronize()
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+
+    binding.calib_index_build(buf, n_end, index)   # the timed update above left the index of a larger fill
+    cold = {
+        "rank_classify_indexed_us": cold_us(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, cfg["alphas"],
+                                                                              numer, p, stage3, counts3)),
+        "rank_classify_us": cold_us(lambda: binding.rank_classify(scores, buf, n_end, cfg["alphas"], numer, p, stage3, counts3)),
+        "classify_us": cold_us(lambda: binding.classify(numer, n_end, 0.1, stage, counts)),
+        "update_indexed_us": cold_us(lambda: binding.calib_update_indexed(buf, n_end, news[0], index, ws)),
+        "note": "L2 flushed by a 512 MB write before each call; one call between two events",
+    }
+    del scrub
     rank_bytes = 12.0 * Nc + 4.0 * n_end
     cls_bytes = 5.0 * Nc
     fused_bytes = rank_bytes + len(cfg["alphas"]) * Nc
@@ -240,7 +284,10 @@ def conformal_stress(torch, binding, peaks):
         "rank_classify_fused_us": ms_fused * 1e3, "rank_classify_fused_gbs": fused_bytes / (ms_fused * 1e-3) / 1e9,
         "rank_classify_indexed_us": ms_fused_ix * 1e3, "rank_classify_indexed_gbs": fused_bytes / (ms_fused_ix * 1e-3) / 1e9,
         "update_indexed_us": ms_upd_ix * 1e3,
+        "cold_l2": cold,
     }
+    if binding.last_device_status() != 0:
+        raise RuntimeError("a conformal kernel reported a device-side error during the benchmark")
     del scores, numer, p, stage, stage3
     out.update(conformal_scaled(torch, binding, peaks, graph_ms))
     return out
@@ -308,7 +355,13 @@ def conformal_scaled(torch, binding, peaks, graph_ms):
     cbytes = 20.0 * ncond    # score + group id in, numer + denom + p out
     out["scaled_rank_conditional"] = {"Nc": ncond, "groups": G, "group_size": m, "us": ms * 1e3,
                                       "gbs": cbytes / (ms * 1e-3) / 1e9, "frac_hbm": cbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-    del sc, nm, pv, st, gid, dn, segs
+    # the same with the candidates of one input adjacent (how a batch of per-input samples arrives)
+    gid_grouped = torch.sort(gid).values
+    ms = graph_ms(lambda: binding.conformal_rank_conditional(sc[:ncond], gid_grouped, segs, seg_off, nm[:ncond], dn, pv[:ncond]), reps=2)
+    out["scaled_rank_conditional_grouped"] = {"Nc": ncond, "groups": G, "group_size": m, "us": ms * 1e3,
+                                              "gbs": cbytes / (ms * 1e-3) / 1e9, "frac_hbm": cbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                              "note": "group ids non-decreasing: candidates of one input are adjacent"}
+    del sc, nm, pv, st, gid, gid_grouped, dn, segs
     n_big = 1 << 22
     bufb = torch.empty(n_big + k, device=dev)
     bufb[:n_big] = torch.sort(torch.randn(n_big, device=dev, generator=gen).exp_()).values
@@ -560,6 +613,7 @@ def run_ours(args):
             line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                     "sample": f"{rows} of {M} token rows of the same batch (full d and V) in {dt:.1f} s, "
                                               f"then rank/classify/update on N={N} scores"}
+            line["cpu_baseline"]["conformal_only"] = oracle_conformal_steps(orc)
         if not args.no_conformal:
             del H_d, W_d
             torch.cuda.empty_cache()

@@ -544,10 +544,12 @@ int atts_conformal_rank_conditional(const float* scores, const int32_t* group_id
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
   if (Nc == 0) return ATTS_OK;
-  int64_t blocks = (Nc + 255) / 256;
+  int64_t blocks = (Nc + 1023) / 1024;
   if (blocks > (int64_t)di->sm_count * 8) blocks = (int64_t)di->sm_count * 8;
+  const bool vec4 = aligned(scores, 16) && aligned(group_ids, 16) && aligned(numer, 16) && aligned(denom, 16) &&
+                    aligned(pvalue, 16);
   rank_conditional_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      scores, group_ids, Nc, calib_segments, seg_offsets, (int)G, numer, denom, pvalue, di->dev_status);
+      scores, group_ids, Nc, calib_segments, seg_offsets, (int)G, numer, denom, pvalue, vec4, di->dev_status);
   return launch_status();
 }
 

@@ -791,34 +791,110 @@ classify_threshold_kernel(const float* __restrict__ scores, int64_t Nc, const fl
 //   numer = 1 + #{own segment >= s},  denom = |segment| + 1,  p = numer / denom;  reject iff
 //   1 <= numer <= floor(alpha * denom)  (evaluated in IEEE double, as on the host for the marginal form).
 // ---------------------------------------------------------------------------------------------
+constexpr int kCondStage = 512;   // calibration entries a warp can stage in shared memory (2 KB)
+
+// Lower bound of four scores in their own segments [lo, lo + len), advanced together so that the dependent loads
+// overlap; `data` is indexed by the same positions as the segments (shared or global memory).
+__device__ __forceinline__ void lower_bound_four(const float* data, const float (&s)[4], int (&lo)[4], int (&len)[4]) {
+  const float qnan = __uint_as_float(0x7FC00000u);
+  while (max(max(len[0], len[1]), max(len[2], len[3])) > 0) {
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = len[e] > 0 ? data[lo[e] + (len[e] >> 1)] : qnan;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (len[e] > 0) {
+        const int half = len[e] >> 1;
+        const bool less = v[e] < s[e];
+        lo[e] = less ? lo[e] + half + 1 : lo[e];
+        len[e] = less ? len[e] - half - 1 : half;
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(256)
 rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restrict__ group_ids, int64_t Nc,
                         const float* __restrict__ calib, const int32_t* __restrict__ seg_offsets, int G,
                         uint32_t* __restrict__ numer, uint32_t* __restrict__ denom, float* __restrict__ pvalue,
-                        unsigned int* __restrict__ dev_status) {
-  for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < Nc; j += (int64_t)gridDim.x * 256) {
-    const float s = scores[j];
-    const int g = group_ids[j];
-    uint32_t num = 0u, den = 1u;
-    if (g < 0 || g >= G) {
-      atomicOr(dev_status, 4u);  // group id out of range: no calibration set, treated as "no score"
+                        bool vec4, unsigned int* __restrict__ dev_status) {
+  // A warp takes 128 consecutive candidates, four per lane (128-bit loads and stores when every array is 16-byte
+  // aligned: vec4).  The candidates of one input usually arrive together, so the segments a warp needs are few
+  // and adjacent: if they span at most kCondStage entries the warp copies that span into shared memory with
+  // coalesced loads and searches there; otherwise every lane searches its segments in global memory.
+  __shared__ float stage_sh[8][kCondStage];
+  const float qnan = __uint_as_float(0x7FC00000u);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* const stage = stage_sh[warp];
+  const int64_t warps_total = (int64_t)gridDim.x * 8;
+  for (int64_t w0 = ((int64_t)blockIdx.x * 8 + warp) * 128; w0 < Nc; w0 += warps_total * 128) {
+    const int64_t j = w0 + 4 * lane;
+    const bool full = vec4 && j + 4 <= Nc;
+    float s[4];
+    int g[4];
+    if (full) {
+      const float4 s4 = *reinterpret_cast<const float4*>(scores + j);
+      const int4 g4 = *reinterpret_cast<const int4*>(group_ids + j);
+      s[0] = s4.x; s[1] = s4.y; s[2] = s4.z; s[3] = s4.w;
+      g[0] = g4.x; g[1] = g4.y; g[2] = g4.z; g[3] = g4.w;
     } else {
-      const int a = __ldg(seg_offsets + g), b = __ldg(seg_offsets + g + 1);
-      den = (uint32_t)(b - a) + 1u;
-      if (s == s) {
-        int lo = a, len = b - a;  // first entry of the segment that is not below s
-        while (len > 0) {
-          const int half = len >> 1;
-          const bool less = __ldg(calib + lo + half) < s;
-          lo = less ? lo + half + 1 : lo;
-          len = less ? len - half - 1 : half;
-        }
-        num = (uint32_t)(b - lo) + 1u;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        s[e] = j + e < Nc ? scores[j + e] : qnan;
+        g[e] = j + e < Nc ? group_ids[j + e] : -1;
       }
     }
-    numer[j] = num;
-    denom[j] = den;
-    if (pvalue) pvalue[j] = num ? __fdiv_rn((float)num, (float)den) : __uint_as_float(0x7FC00000u);
+    int lo[4], len[4], end[4];
+    uint32_t den[4];
+    bool bad = false;
+    int span_lo = 0x7FFFFFFF, span_hi = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool ok = g[e] >= 0 && g[e] < G;
+      bad = bad || (!ok && j + e < Nc);
+      const int a = ok ? __ldg(seg_offsets + g[e]) : 0, b = ok ? __ldg(seg_offsets + g[e] + 1) : 0;
+      lo[e] = a;
+      end[e] = b;
+      den[e] = ok ? (uint32_t)(b - a) + 1u : 1u;
+      len[e] = (ok && s[e] == s[e]) ? b - a : -1;   // -1: no score (NaN, or no calibration set)
+      if (len[e] > 0) {
+        span_lo = min(span_lo, a);
+        span_hi = max(span_hi, b);
+      }
+    }
+    if (bad) atomicOr(dev_status, 4u);  // group id out of range: no calibration set, treated as "no score"
+    const bool scored[4] = {len[0] >= 0, len[1] >= 0, len[2] >= 0, len[3] >= 0};
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      span_lo = min(span_lo, __shfl_xor_sync(0xFFFFFFFFu, span_lo, o));
+      span_hi = max(span_hi, __shfl_xor_sync(0xFFFFFFFFu, span_hi, o));
+    }
+    if (span_hi - span_lo <= kCondStage) {   // warp-uniform (an empty span gives a negative difference)
+      __syncwarp();                          // the previous round's searches are done with the staging area
+      for (int t = span_lo + lane; t < span_hi; t += 32) stage[t - span_lo] = __ldg(calib + t);
+      __syncwarp();
+      lower_bound_four(stage - span_lo, s, lo, len);
+    } else {
+      lower_bound_four(calib, s, lo, len);
+    }
+    uint32_t num[4];
+    float p[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      num[e] = scored[e] ? (uint32_t)(end[e] - lo[e]) + 1u : 0u;
+      p[e] = num[e] ? __fdiv_rn((float)num[e], (float)den[e]) : qnan;
+    }
+    if (full) {
+      *reinterpret_cast<uint4*>(numer + j) = make_uint4(num[0], num[1], num[2], num[3]);
+      *reinterpret_cast<uint4*>(denom + j) = make_uint4(den[0], den[1], den[2], den[3]);
+      if (pvalue) *reinterpret_cast<float4*>(pvalue + j) = make_float4(p[0], p[1], p[2], p[3]);
+    } else {
+      for (int e = 0; e < 4 && j + e < Nc; ++e) {
+        numer[j + e] = num[e];
+        denom[j + e] = den[e];
+        if (pvalue) pvalue[j + e] = p[e];
+      }
+    }
   }
 }
 

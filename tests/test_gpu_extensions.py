@@ -75,6 +75,18 @@ def test_conditional_rank_and_classify_bit_exact():
     binding.conformal_rank_conditional(dev(scores), dev(gid2), dev(calib), dev(off), numer, denom, None)
     assert binding.last_device_status() & binding.DEV_GROUP_ID_RANGE
     assert host_u32(numer)[10] == 0
+    # ragged tails and arrays that are not 16-byte aligned take the scalar loads and stores
+    for start, stop in ((0, Nc - 1), (1, Nc), (3, Nc - 2), (0, 3)):
+        m = stop - start
+        numer3, denom3, p3 = poison((m + 4,), torch.int32), poison((m + 4,), torch.int32), poison((m + 4,), torch.float32)
+        shift = start % 4
+        binding.conformal_rank_conditional(dev(scores)[start:stop], dev(gid)[start:stop], dev(calib), dev(off),
+                                           numer3[shift:shift + m], denom3[shift:shift + m], p3[shift:shift + m])
+        assert np.array_equal(host_u32(numer3)[shift:shift + m], want_numer[start:stop])
+        assert np.array_equal(host_u32(denom3)[shift:shift + m], want_denom[start:stop])
+        assert np.array_equal(f32_bits(p3)[shift:shift + m], f32_bits(want_p[start:stop]))
+        assert np.all(host_u32(numer3)[shift + m:] == 0xFFFFFFFF) and np.all(host_u32(numer3)[:shift] == 0xFFFFFFFF)
+    assert binding.last_device_status() == 0
 
 
 @pytest.mark.parametrize("M,d,V", [(300, 192, 1000), (1000, 512, 5000), (4096, 1024, 8192)])
