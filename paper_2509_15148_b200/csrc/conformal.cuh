@@ -795,12 +795,13 @@ constexpr int kCondStage = 512;   // calibration entries a warp can stage in sha
 
 // Lower bound of four scores in their own segments [lo, lo + len), advanced together so that the dependent loads
 // overlap; `data` is indexed by the same positions as the segments (shared or global memory).
+template <bool GLOBAL>
 __device__ __forceinline__ void lower_bound_four(const float* data, const float (&s)[4], int (&lo)[4], int (&len)[4]) {
   const float qnan = __uint_as_float(0x7FC00000u);
   while (max(max(len[0], len[1]), max(len[2], len[3])) > 0) {
     float v[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = len[e] > 0 ? data[lo[e] + (len[e] >> 1)] : qnan;
+    for (int e = 0; e < 4; ++e) v[e] = len[e] > 0 ? (GLOBAL ? __ldg(data + lo[e] + (len[e] >> 1)) : data[lo[e] + (len[e] >> 1)]) : qnan;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       if (len[e] > 0) {
@@ -873,9 +874,9 @@ rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restr
       __syncwarp();                          // the previous round's searches are done with the staging area
       for (int t = span_lo + lane; t < span_hi; t += 32) stage[t - span_lo] = __ldg(calib + t);
       __syncwarp();
-      lower_bound_four(stage - span_lo, s, lo, len);
+      lower_bound_four<false>(stage - span_lo, s, lo, len);
     } else {
-      lower_bound_four(calib, s, lo, len);
+      lower_bound_four<true>(calib, s, lo, len);
     }
     uint32_t num[4];
     float p[4];
