@@ -127,3 +127,52 @@ def test_conformal_stress_at_maximum_buffer_size():
     n2 = binding.calib_update(buf, n, dev(new), workspace(binding.calib_workspace_bytes(n, k)))
     assert n2 == n + k
     assert np.array_equal(f32_bits(buf), f32_bits(orc.calib_update(calib, new)))
+
+
+def test_conformal_stress_whole_sequence_with_index_in_one_graph():
+    """The conformal-only workload in the form the benchmark times: all 64 steps (rank + three alphas through the
+    calibration index, then the indexed update) captured in one CUDA graph and replayed.  The last step's ranks,
+    p-values, stages and counts and the final buffer are compared with the oracle, which replays the 64 inserts."""
+    cfg = inputs.CONFORMAL_STRESS
+    Nc, n0, k, steps, alphas = cfg["Nc"], cfg["n0"], cfg["k"], cfg["steps"], cfg["alphas"]
+    scores = inputs.lognormal_scores(inputs.BASE_SEED + 1, Nc)
+    calib0 = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, n0))
+    news_h = [inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, k) for t in range(steps)]
+    cap = n0 + k * steps
+    s_dev, c0_dev, news = dev(scores), dev(calib0), [dev(x) for x in news_h]
+    buf = poison((cap,), torch.float32)
+    numer, p = poison((Nc,), torch.int32), poison((Nc,), torch.float32)
+    stage, counts = poison((len(alphas), Nc), torch.uint8), poison((len(alphas), 3), torch.int32)
+    index = workspace(binding.calib_index_bytes(cap))
+    ws = workspace(binding.calib_workspace_bytes(cap, k))
+
+    def sequence():
+        buf[:n0] = c0_dev
+        binding.calib_index_build(buf, n0, index)
+        n = n0
+        for t in range(steps):
+            binding.rank_classify_indexed(s_dev, buf, n, index, alphas, numer, p, stage, counts)
+            n = binding.calib_update_indexed(buf, n, news[t], index, ws)
+        return n
+
+    assert sequence() == cap                       # eager once (also the device set-up)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        sequence()
+    for t in (numer, p, stage, counts):
+        t.view(torch.uint8).fill_(0xFF)
+    g.replay()
+    torch.cuda.synchronize()
+    calib = calib0
+    for t in range(steps - 1):
+        calib = orc.calib_update(calib, news_h[t])
+    want_numer = orc.conformal_numer_sorted(scores, calib)     # the last step ranks against n = cap - k entries
+    assert np.array_equal(host_u32(numer), want_numer)
+    assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, calib.size)))
+    for a, alpha in enumerate(alphas):
+        want_stage, want_counts = orc.classify(want_numer, calib.size, alpha)
+        assert np.array_equal(stage[a].cpu().numpy(), want_stage)
+        assert np.array_equal(host_u32(counts[a]), want_counts)
+    assert np.array_equal(f32_bits(buf), f32_bits(orc.calib_update(calib, news_h[-1])))
+    assert binding.last_device_status() == 0
