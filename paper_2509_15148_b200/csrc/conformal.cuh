@@ -282,7 +282,7 @@ rank_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restric
 // ---------------------------------------------------------------------------------------------
 constexpr int kBucketMaxN = 8191;
 constexpr int kBucketMaxLog2 = 15;   // at most 32768 buckets (128 KB)
-constexpr int kBucketPad = 2;        // NaN entries behind the buffer copy, so probes need no bounds check
+constexpr int kBucketPad = 2;        // NaN entries behind the buffer copy (no probe can leave the array)
 constexpr int64_t kBucketMinCandidates = 1 << 16;
 
 struct BucketMap {
