@@ -175,6 +175,17 @@ def classify(numer: np.ndarray, n: int, alpha: float):
     return stage, counts
 
 
+def takeover_ids(stage: np.ndarray) -> np.ndarray:
+    """The samples the target model takes over in this turn ("Budget Prediction", Sec. 3.2: the B candidates that
+    are rejected; "Target Sampling", Sec. 3.3: the candidates the target continues): the positions whose stage is 3,
+    in input order.  Their number is the budget B."""
+    out = []
+    for j, st in enumerate(np.asarray(stage, dtype=np.uint8).tolist()):
+        if st == STAGE_TARGET:
+            out.append(j)
+    return np.array(out, dtype=np.int32)
+
+
 def calib_update(calib_sorted: np.ndarray, new_scores: np.ndarray) -> np.ndarray:
     """Online calibration: the set grows by the new scores and stays ascending (Sec. 3.2).
 

@@ -85,3 +85,23 @@ def test_rms_inv_and_scaled_logprob_match_torch_rms_norm():
     # scale 1 is the unscaled function; a scale that sends logits to zero gives the uniform distribution
     np.testing.assert_allclose(orc.token_logprob_scaled(Hb, Wb, ids, np.ones(M)), orc.token_logprob(Hb, Wb, ids), atol=1e-13)
     np.testing.assert_allclose(orc.token_logprob_scaled(Hb, Wb, ids, np.zeros(M)), -math.log(V), atol=1e-13)
+
+
+def test_takeover_ids_hand_example_library_routine_and_budget():
+    # worked by hand: stages 2 3 1 3 3 2 -> the target takes over samples 1, 3 and 4; B = 3
+    assert orc.takeover_ids(np.array([2, 3, 1, 3, 3, 2], np.uint8)).tolist() == [1, 3, 4]
+    assert orc.takeover_ids(np.zeros(0, np.uint8)).size == 0
+    assert orc.takeover_ids(np.array([1, 2, 2], np.uint8)).size == 0
+    # against a library routine, and against the count classify reports as the budget
+    calib = np.sort(inputs.lognormal_scores(5, 999))
+    s = inputs.lognormal_scores(6, 5000)
+    s[::97] = np.nan
+    for alpha in (0.05, 0.25, 0.6):
+        stage, counts = orc.classify(orc.conformal_numer_sorted(s, calib), calib.size, alpha)
+        ids = orc.takeover_ids(stage)
+        assert np.array_equal(ids, torch.nonzero(torch.from_numpy(stage) == 3).flatten().numpy())
+        assert ids.size == counts[2]
+        assert np.all(np.diff(ids) > 0)
+        # exactly the samples with p <= alpha (Eq. prediction_set's complement), none without a score
+        p = orc.pvalue(orc.conformal_numer_sorted(s, calib), calib.size)
+        assert set(ids.tolist()) == {j for j in range(s.size) if p[j] <= alpha}
