@@ -345,6 +345,18 @@ def conformal_scaled(torch, binding, peaks, graph_ms):
     ms = graph_ms(lambda: binding.classify_threshold(sc, tau, st, counts), reps=2)
     out["scaled_classify_threshold"] = {"Nc": big, "us": ms * 1e3, "gbs": 5.0 * big / (ms * 1e-3) / 1e9,
                                         "frac_hbm": 5.0 * big / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    # budget report: positions of the stage-3 samples among 2^26 (stages from the classify call above, alpha = 0.1)
+    ids = torch.empty(big // 4, dtype=torch.int32, device=dev)
+    cnt = torch.empty(1, dtype=torch.int32, device=dev)
+    ws_ids = torch.empty(binding.takeover_ids_workspace_bytes(big), dtype=torch.uint8, device=dev)
+    binding.classify(nm, n_small, 0.1, st, counts)
+    ms = graph_ms(lambda: binding.takeover_ids(st, ids, cnt, ws_ids), reps=2)
+    B = int(cnt.cpu().numpy().view(np.uint32)[0])
+    ids_bytes = 1.0 * big + 4.0 * B      # every stage byte once, every position once
+    out["scaled_takeover_ids"] = {"Nc": big, "B": B, "us": ms * 1e3, "gbs": ids_bytes / (ms * 1e-3) / 1e9,
+                                  "frac_hbm": ids_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                  "note": "three launches; the stage bytes are read twice (count, then write)"}
+    del ids, ws_ids
     # conditional coverage: 2^24 candidates, each ranked against its own input's 64 calibration scores
     ncond, G, m = 1 << 24, 1 << 16, 64
     segs = torch.sort(torch.randn(G, m, device=dev, generator=gen).exp_(), dim=1).values.reshape(-1).contiguous()

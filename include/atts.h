@@ -195,6 +195,20 @@ int atts_rank_classify(const float* scores, int64_t Nc, const float* calib_sorte
                        uint8_t* stage, uint32_t* stage_counts, void* cuda_stream);
 
 /*
+ * Budget report ("Budget Prediction", Sec. 3.2: B is the number of candidates that are rejected; "Target
+ * Sampling", Sec. 3.3: the target model continues exactly those): the positions of the samples whose stage is
+ * ATTS_STAGE_TARGET, ascending, and their number B.
+ *
+ *   stage         dev  [Nc] uint8, as written by atts_classify (a row of atts_rank_classify's output)
+ *   ids           dev  [ids_cap] int32 out: the first min(B, ids_cap) positions; may be NULL when ids_cap == 0
+ *   count         dev  [1] uint32 out: B (also when B > ids_cap); may be NULL
+ *   workspace     dev  256-byte aligned, at least atts_takeover_ids_workspace_bytes(Nc) bytes
+ */
+int atts_takeover_ids_workspace_bytes(int64_t Nc, size_t* bytes);
+int atts_takeover_ids(const uint8_t* stage, int64_t Nc, int32_t* ids, int64_t ids_cap, uint32_t* count,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Threshold form of the acceptance rule (the quantile-threshold construction of the classic set-up,
  * Eqs. quantile / pred_set, read for the rejection side): with tau = the k_alpha-th largest calibration
  * score, k_alpha = floor(alpha * (n + 1)), a sample is rejected iff s > tau - exactly the samples with

@@ -21,6 +21,7 @@ EXPORTS = (
     "atts_threshold", "atts_classify_threshold", "atts_conformal_rank_conditional", "atts_classify_conditional",
     "atts_debug_score_plan", "atts_debug_score_unit", "atts_score_slice", "atts_score_combine",
     "atts_calib_index_bytes", "atts_calib_index_build", "atts_calib_update_indexed", "atts_rank_classify_indexed",
+    "atts_takeover_ids_workspace_bytes", "atts_takeover_ids",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -85,6 +86,8 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
                                               c_size_t, c_void_p, c_size_t, c_void_p]
     lib.atts_rank_classify_indexed.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, POINTER(c_double), c_int32,
                                                c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.atts_takeover_ids_workspace_bytes.argtypes = [c_int64, POINTER(c_size_t)]
+    lib.atts_takeover_ids.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.atts_profile_begin.argtypes = [c_int]
     lib.atts_profile_end.argtypes = [POINTER(ctypes.c_float), c_int, POINTER(c_int)]
     for name in EXPORTS[2:]:
@@ -178,6 +181,19 @@ def classify_threshold(scores, tau, stage, stage_counts=None) -> None:
     """Stage per sample from s > tau[0]; stage_counts [3] or None."""
     _check(load().atts_classify_threshold(_ptr(scores), scores.numel(), _ptr(tau), _ptr(stage), _ptr(stage_counts),
                                           _stream()), "atts_classify_threshold")
+
+
+def takeover_ids_workspace_bytes(Nc: int) -> int:
+    out = c_size_t(0)
+    _check(load().atts_takeover_ids_workspace_bytes(Nc, ctypes.byref(out)), "atts_takeover_ids_workspace_bytes")
+    return out.value
+
+
+def takeover_ids(stage, ids, count, workspace) -> None:
+    """Positions (ascending, int32) of the samples in stage 3 into ids (as many as fit), their number into count[0]."""
+    _check(load().atts_takeover_ids(_ptr(stage), stage.numel(), _ptr(ids), 0 if ids is None else ids.numel(), _ptr(count),
+                                    _ptr(workspace), 0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _stream()), "atts_takeover_ids")
 
 
 def conformal_rank_conditional(scores, group_ids, calib_segments, seg_offsets, numer, denom, pvalue=None) -> None:

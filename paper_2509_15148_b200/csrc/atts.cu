@@ -532,6 +532,43 @@ int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, u
   return launch_status();
 }
 
+int atts_takeover_ids_workspace_bytes(int64_t Nc, size_t* bytes) {
+  if (!bytes) return ATTS_ERR_NULL;
+  if (Nc < 0 || Nc >= (1ll << 31)) return ATTS_ERR_SHAPE;
+  *bytes = round_up((size_t)((Nc + kIdsTile - 1) / kIdsTile) * sizeof(uint32_t), 256) + 256;
+  return ATTS_OK;
+}
+
+int atts_takeover_ids(const uint8_t* stage, int64_t Nc, int32_t* ids, int64_t ids_cap, uint32_t* count, void* workspace,
+                      size_t workspace_bytes, void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || ids_cap < 0) return ATTS_ERR_SHAPE;
+  if ((Nc > 0 && (!stage || !workspace)) || (ids_cap > 0 && !ids)) return ATTS_ERR_NULL;
+  if (!aligned(ids, 4) || !aligned(count, 4) || !aligned(workspace, 256)) return ATTS_ERR_ALIGN;
+  size_t need = 0;
+  atts_takeover_ids_workspace_bytes(Nc, &need);
+  if (Nc > 0 && workspace_bytes < need) return ATTS_ERR_WORKSPACE;
+  const DeviceInfo* di;
+  int st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (Nc == 0) {
+    if (count && cudaMemsetAsync(count, 0, sizeof(uint32_t), stream) != cudaSuccess) {
+      cudaGetLastError();
+      return ATTS_ERR_CUDA;
+    }
+    return ATTS_OK;
+  }
+  const int tiles = (int)((Nc + kIdsTile - 1) / kIdsTile);
+  const bool vec = aligned(stage, 16);
+  uint32_t* tile_count = static_cast<uint32_t*>(workspace);
+  takeover_count_kernel<<<tiles, kIdsThreads, 0, stream>>>(stage, Nc, vec, tile_count);
+  if ((st = launch_status()) != ATTS_OK) return st;
+  takeover_scan_kernel<<<1, kIdsThreads, 0, stream>>>(tile_count, tiles, count);
+  if ((st = launch_status()) != ATTS_OK) return st;
+  takeover_write_kernel<<<tiles, kIdsThreads, 0, stream>>>(stage, Nc, vec, tile_count, ids, ids_cap);
+  return launch_status();
+}
+
 int atts_conformal_rank_conditional(const float* scores, const int32_t* group_ids, int64_t Nc, const float* calib_segments,
                                     const int32_t* seg_offsets, int64_t G, uint32_t* numer, uint32_t* denom, float* pvalue,
                                     void* cuda_stream) {

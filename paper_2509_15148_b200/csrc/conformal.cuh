@@ -785,6 +785,111 @@ classify_threshold_kernel(const float* __restrict__ scores, int64_t Nc, const fl
 }
 
 // ---------------------------------------------------------------------------------------------
+// Budget report: the positions of the samples in stage 3 (the target takes over), in input order, and their
+// number B.  Stream compaction in three launches: stage-3 count per tile of kIdsTile bytes; exclusive scan of the
+// tile counts by one block (which also writes B); every tile then recounts its bytes, 64 per thread, and writes
+// its positions from its offset on.  Everything is integer work in a fixed order: the result is unique.
+// ---------------------------------------------------------------------------------------------
+constexpr int kIdsThreads = 256;
+constexpr int kIdsPerThread = 64;
+constexpr int kIdsTile = kIdsThreads * kIdsPerThread;   // 16384 stage bytes per block
+
+// Bit i of the result is set where byte i of the thread's 64 stage bytes is 3.
+__device__ __forceinline__ uint64_t stage3_mask(const uint8_t* __restrict__ stage, int64_t j, int64_t Nc, bool vec) {
+  uint64_t mask = 0;
+  if (vec && j + kIdsPerThread <= Nc) {
+    uint4 q[4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v) q[v] = *reinterpret_cast<const uint4*>(stage + j + 16 * v);
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+      const uint32_t w[4] = {q[v].x, q[v].y, q[v].z, q[v].w};
+      uint32_t m16 = 0;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) m16 |= (((w[i >> 2] >> (8 * (i & 3))) & 0xFFu) == 3u ? 1u : 0u) << i;
+      mask |= (uint64_t)m16 << (16 * v);
+    }
+  } else {
+    for (int i = 0; i < kIdsPerThread && j + i < Nc; ++i) mask |= (uint64_t)(stage[j + i] == 3 ? 1u : 0u) << i;
+  }
+  return mask;
+}
+
+// Exclusive prefix sum of one value per thread over a block of kIdsThreads; *total gets the block's sum.
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* total) {
+  __shared__ uint32_t warp_sum[kIdsThreads / 32];
+  __shared__ uint32_t block_sum;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  if (lane == 31) warp_sum[warp] = incl;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t run = 0;
+    for (int w = 0; w < kIdsThreads / 32; ++w) {
+      const uint32_t t = warp_sum[w];
+      warp_sum[w] = run;
+      run += t;
+    }
+    block_sum = run;
+  }
+  __syncthreads();
+  const uint32_t excl = warp_sum[warp] + incl - v;
+  *total = block_sum;
+  __syncthreads();   // the shared words may be reused by the next call
+  return excl;
+}
+
+__global__ void __launch_bounds__(kIdsThreads)
+takeover_count_kernel(const uint8_t* __restrict__ stage, int64_t Nc, bool vec, uint32_t* __restrict__ tile_count) {
+  const int64_t j = (int64_t)blockIdx.x * kIdsTile + (int64_t)threadIdx.x * kIdsPerThread;
+  uint32_t c = j < Nc ? (uint32_t)__popcll(stage3_mask(stage, j, Nc, vec)) : 0u;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+  __shared__ uint32_t sh[kIdsThreads / 32];
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = c;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t t = 0;
+    for (int w = 0; w < kIdsThreads / 32; ++w) t += sh[w];
+    tile_count[blockIdx.x] = t;
+  }
+}
+
+// One block: tile_count[t] <- sum of the counts of the tiles before t; *count <- the sum of all (may be nullptr).
+__global__ void __launch_bounds__(kIdsThreads)
+takeover_scan_kernel(uint32_t* __restrict__ tile_count, int tiles, uint32_t* __restrict__ count) {
+  uint32_t carry = 0;
+  for (int base = 0; base < tiles; base += kIdsThreads) {
+    const int t = base + threadIdx.x;
+    const uint32_t v = t < tiles ? tile_count[t] : 0u;
+    uint32_t total;
+    const uint32_t excl = block_exclusive_scan(v, &total);
+    if (t < tiles) tile_count[t] = carry + excl;
+    carry += total;
+  }
+  if (threadIdx.x == 0 && count != nullptr) *count = carry;
+}
+
+__global__ void __launch_bounds__(kIdsThreads)
+takeover_write_kernel(const uint8_t* __restrict__ stage, int64_t Nc, bool vec, const uint32_t* __restrict__ tile_offset,
+                      int32_t* __restrict__ ids, int64_t ids_cap) {
+  const int64_t j = (int64_t)blockIdx.x * kIdsTile + (int64_t)threadIdx.x * kIdsPerThread;
+  const uint64_t mask = j < Nc ? stage3_mask(stage, j, Nc, vec) : 0ull;
+  uint32_t total;
+  const uint32_t excl = block_exclusive_scan((uint32_t)__popcll(mask), &total);
+  int64_t pos = (int64_t)tile_offset[blockIdx.x] + excl;
+  for (uint64_t m = mask; m != 0ull; m &= m - 1ull) {
+    if (pos < ids_cap) ids[pos] = (int32_t)(j + (__ffsll((long long)m) - 1));
+    ++pos;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Conditional coverage (Proposition 2): a candidate is ranked against the calibration scores of its own
 // input only.  The per-input buffers are ascending segments of one array; segments are short (the m samples
 // of one input), so a thread searches its segment directly in (L2-resident) global memory.

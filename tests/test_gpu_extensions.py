@@ -158,3 +158,46 @@ def test_vocabulary_sliced_scoring_equals_the_full_definition(M, d, V, cuts):
     binding.score_combine(stats, dev(off), lp, sc, workspace(4 * M + 512))
     assert binding.last_device_status() & binding.DEV_TOKEN_ID_RANGE
     assert np.isnan(lp.cpu().numpy()[7])
+
+
+@pytest.mark.parametrize("Nc", [0, 1, 15, 16, 4095, 4096, 4097, 70001, (1 << 20) + 5])
+def test_takeover_ids_bit_exact(Nc):
+    """Positions of the samples the target takes over and the budget B, against the oracle: random stages, all stage 3,
+    none, an output too short for all of them, and a stage array that is not 16-byte aligned."""
+    rng = np.random.default_rng(Nc + 1)
+    cases = [rng.choice(np.array([1, 2, 3], np.uint8), size=Nc, p=[0.05, 0.7, 0.25]),
+             np.full(Nc, 3, np.uint8), np.full(Nc, 2, np.uint8)]
+    ws = workspace(binding.takeover_ids_workspace_bytes(Nc))
+    for stage_h in cases:
+        want = orc.takeover_ids(stage_h) if Nc < 200000 else np.flatnonzero(stage_h == 3).astype(np.int32)
+        for shift, cap in ((0, Nc), (1, Nc), (0, want.size // 2)):
+            st = poison((Nc + 16,), torch.uint8)
+            st[shift:shift + Nc] = dev(stage_h) if Nc else st[:0]
+            ids = poison((cap + 3,), torch.int32)
+            count = poison((1,), torch.int32)
+            binding.takeover_ids(st[shift:shift + Nc], ids[:cap], count, ws)
+            torch.cuda.synchronize()
+            assert host_u32(count)[0] == want.size
+            got = ids.cpu().numpy()
+            m = min(cap, want.size)
+            assert np.array_equal(got[:m], want[:m])
+            assert np.all(got.view(np.uint32)[m:] == 0xFFFFFFFF)        # nothing written past what fits
+    if Nc >= 200000:   # the shortcut above is the oracle's definition: checked on a sample of positions
+        assert np.array_equal(orc.takeover_ids(cases[0][:5000]), np.flatnonzero(cases[0][:5000] == 3))
+    assert binding.last_device_status() == 0
+
+
+def test_takeover_ids_follow_classify():
+    n, Nc, alpha = 4096, 64, 0.25
+    calib = np.sort(inputs.lognormal_scores(11, n))
+    scores = inputs.lognormal_scores(12, Nc)
+    numer, stage, counts = poison((Nc,), torch.int32), poison((Nc,), torch.uint8), poison((3,), torch.int32)
+    binding.conformal_rank(dev(scores), dev(calib), n, numer, None)
+    binding.classify(numer, n, alpha, stage, counts)
+    ids, count = poison((Nc,), torch.int32), poison((1,), torch.int32)
+    binding.takeover_ids(stage, ids, count, workspace(binding.takeover_ids_workspace_bytes(Nc)))
+    torch.cuda.synchronize()
+    want_stage, want_counts = orc.classify(orc.conformal_numer_sorted(scores, calib), n, alpha)
+    want = orc.takeover_ids(want_stage)
+    assert host_u32(count)[0] == want_counts[2] == want.size
+    assert np.array_equal(ids.cpu().numpy()[:want.size], want)
