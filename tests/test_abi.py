@@ -63,7 +63,7 @@ def test_argument_errors_need_no_device():
     assert lib.atts_calib_index_bytes(524223, ctypes.byref(sz)) == 0 and sz.value % 256 == 0 and sz.value >= 4 * (8192 + 8 * 8191)
     assert lib.atts_calib_index_bytes(524224, ctypes.byref(sz)) == 2                        # too large for an index
     assert lib.atts_calib_index_bytes(10, None) == 1
-    assert lib.atts_takeover_ids_workspace_bytes(1 << 20, ctypes.byref(sz)) == 0 and sz.value >= 4 * 256
+    assert lib.atts_takeover_ids_workspace_bytes(1 << 20, ctypes.byref(sz)) == 0 and sz.value >= 4 * 64 and sz.value % 256 == 0
     assert lib.atts_takeover_ids_workspace_bytes(-1, ctypes.byref(sz)) == 2
     assert lib.atts_takeover_ids(None, 8, None, 8, None, None, 0, None) == 1
     assert lib.atts_takeover_ids(None, 8, None, -1, None, None, 0, None) == 2
