@@ -975,7 +975,8 @@ rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restr
       span_lo = min(span_lo, __shfl_xor_sync(0xFFFFFFFFu, span_lo, o));
       span_hi = max(span_hi, __shfl_xor_sync(0xFFFFFFFFu, span_hi, o));
     }
-    if (span_hi - span_lo <= kCondStage) {   // warp-uniform (an empty span gives a negative difference)
+    // warp-uniform; no candidate of the warp with anything to search leaves span_lo above span_hi: nothing is staged
+    if (span_hi > span_lo && span_hi - span_lo <= kCondStage) {
       __syncwarp();                          // the previous round's searches are done with the staging area
       for (int t = span_lo + lane; t < span_hi; t += 32) stage[t - span_lo] = __ldg(calib + t);
       __syncwarp();

@@ -89,6 +89,30 @@ def test_conditional_rank_and_classify_bit_exact():
     assert binding.last_device_status() == 0
 
 
+def test_conditional_rank_warps_with_nothing_to_search():
+    """Whole warps whose candidates have no entries to search: empty calibration sets, scores that are all NaN, and a
+    single group; then a mix in which only some warps have work."""
+    def run(scores, gid, groups):
+        off = np.concatenate([[0], np.cumsum([len(x) for x in groups])]).astype(np.int32)
+        calib = np.concatenate(groups).astype(np.float32) if off[-1] else np.zeros(1, np.float32)
+        Nc = scores.size
+        numer, denom, p = poison((Nc,), torch.int32), poison((Nc,), torch.int32), poison((Nc,), torch.float32)
+        binding.conformal_rank_conditional(dev(scores), dev(gid), dev(calib), dev(off), numer, denom, p)
+        torch.cuda.synchronize()
+        wn, wd = orc.conformal_numer_conditional(scores, gid, groups)
+        assert np.array_equal(host_u32(numer), wn) and np.array_equal(host_u32(denom), wd)
+
+    empty = np.zeros(0, np.float32)
+    scores = inputs.lognormal_scores(21, 1000)
+    run(scores, np.zeros(1000, np.int32), [empty])                                   # one group, no calibration scores
+    run(scores, (np.arange(1000) % 5).astype(np.int32), [empty] * 5)                 # every group empty
+    run(np.full(1000, np.nan, np.float32), np.zeros(1000, np.int32), [np.sort(inputs.lognormal_scores(22, 40))])
+    groups = [empty, np.sort(inputs.lognormal_scores(23, 30)), empty, np.sort(inputs.lognormal_scores(24, 700))]
+    gid = np.sort(np.random.default_rng(5).integers(0, 4, size=3000)).astype(np.int32)
+    run(inputs.lognormal_scores(25, 3000), gid, groups)                              # warps of empty and of large groups
+    assert binding.last_device_status() == 0
+
+
 @pytest.mark.parametrize("M,d,V", [(300, 192, 1000), (1000, 512, 5000), (4096, 1024, 8192)])
 def test_rms_inv_and_scaled_scoring(M, d, V):
     rng = np.random.default_rng(M)
