@@ -225,3 +225,38 @@ def test_takeover_ids_follow_classify():
     want = orc.takeover_ids(want_stage)
     assert host_u32(count)[0] == want_counts[2] == want.size
     assert np.array_equal(ids.cpu().numpy()[:want.size], want)
+
+
+def test_conditional_rank_randomised_groups_and_alignments():
+    """Sixty random problems: group counts and sizes from empty to thousands of entries (staged and unstaged warps),
+    sorted and shuffled group ids, rounded values (ties), a NaN score, and output arrays at every 4-byte alignment."""
+    rng = np.random.default_rng(20250131)
+    for case in range(60):
+        G = int(rng.choice([1, 2, 7, 100, 3000]))
+        sizes = rng.integers(0, int(rng.choice([1, 8, 64, 600, 3000])) + 1, size=G)
+        digits = int(rng.integers(0, 4))
+        groups = [np.sort(np.round(inputs.lognormal_scores(5000 + 100 * case + g % 97, int(z)), digits)) for g, z in enumerate(sizes)]
+        off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+        calib = np.concatenate(groups).astype(np.float32) if off[-1] else np.zeros(1, np.float32)
+        Nc = int(rng.choice([1, 5, 127, 128, 129, 5000, 40001]))
+        gid = rng.integers(0, G, size=Nc).astype(np.int32)
+        if rng.random() < 0.6:
+            gid = np.sort(gid)
+        scores = np.round(inputs.lognormal_scores(9000 + case, Nc), digits)
+        if Nc > 3:
+            scores[int(rng.integers(0, Nc))] = np.nan
+        shift = int(rng.integers(0, 4))
+        numer, denom, p = poison((Nc + 4,), torch.int32), poison((Nc + 4,), torch.int32), poison((Nc + 4,), torch.float32)
+        s, g = poison((Nc + 4,), torch.float32), poison((Nc + 4,), torch.int32)
+        s[shift:shift + Nc] = dev(scores)
+        g[shift:shift + Nc] = dev(gid)
+        binding.conformal_rank_conditional(s[shift:shift + Nc], g[shift:shift + Nc], dev(calib), dev(off),
+                                           numer[shift:shift + Nc], denom[shift:shift + Nc], p[shift:shift + Nc])
+        torch.cuda.synchronize()
+        wn, wd = orc.conformal_numer_conditional(scores, gid, groups)
+        assert np.array_equal(host_u32(numer)[shift:shift + Nc], wn), (case, G, Nc, shift)
+        assert np.array_equal(host_u32(denom)[shift:shift + Nc], wd), (case, G, Nc, shift)
+        wp = (wn.astype(np.float64) / wd.astype(np.float64)).astype(np.float32)
+        wp[wn == 0] = np.nan
+        assert np.array_equal(f32_bits(p)[shift:shift + Nc], f32_bits(wp)), (case, G, Nc, shift)
+    assert binding.last_device_status() == 0
