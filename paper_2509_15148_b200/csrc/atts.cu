@@ -684,7 +684,7 @@ static int calib_update_impl(float* calib, int64_t n, int64_t cap, const float* 
   int64_t cur = n;
   for (int64_t off = 0; off < k; off += kSortMaxK) {
     const int kc = (int)((k - off) < kSortMaxK ? (k - off) : kSortMaxK);
-    int sort_blocks = (kc + 7) / 8;
+    int sort_blocks = (kc + kSortKeysPerBlock - 1) / kSortKeysPerBlock;
     if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
     sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)((kc + 127) & ~127) * 4, stream>>>(new_scores + off, kc, sorted_keys);
     if ((st = launch_status()) != ATTS_OK) return st;
@@ -735,7 +735,7 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
   uint32_t* sorted_keys = reinterpret_cast<uint32_t*>(scratch);
   float* merged = reinterpret_cast<float*>(scratch + 4 * ATTS_STATIC_MAX_NEW);
   const int kc = (int)k;
-  int sort_blocks = (kc + 7) / 8;
+  int sort_blocks = (kc + kSortKeysPerBlock - 1) / kSortKeysPerBlock;
   if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
   sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)((kc + 127) & ~127) * 4, stream>>>(new_scores, kc, sorted_keys);
   if ((st = launch_status()) != ATTS_OK) return st;

@@ -632,46 +632,55 @@ classify_kernel(const uint32_t* __restrict__ numer, int64_t Nc, uint32_t k_alpha
 
 // ---------------------------------------------------------------------------------------------
 // K5  sort of the new calibration scores by all-pairs ranking, spread over the whole GPU.  Every block
-// holds all k keys in shared memory (padded to a multiple of 128 with a key above every canonical key);
-// one warp per element counts, four keys per 128-bit load, the keys below it and the keys not above it.
-// If only the element itself is equal to it, the first count is its slot; otherwise (ties, rare) the
-// warp also counts the equal keys that come before it in the input, so every element gets its own slot.
-// k is at most kSortMaxK per launch.
+// holds all k keys in shared memory (padded to a multiple of 128 with a key above every canonical key).
+// The slot of key j is the number of keys that sort before it: smaller keys, and equal keys that come earlier
+// in the input - one comparison per pair, key_i < key_j + (i < j).  A warp ranks four consecutive keys at a
+// time, so a 128-bit load of four other keys serves sixteen comparisons; those four others all come before or
+// all come after the warp's four, except in the one group that holds them.  k is at most kSortMaxK per launch.
 // ---------------------------------------------------------------------------------------------
 constexpr int kSortMaxK = 16384;
 constexpr int kSortThreads = 256;
+constexpr int kSortKeysPerBlock = (kSortThreads / 32) * 4;
 
 __global__ void __launch_bounds__(kSortThreads)
 sort_new_kernel(const float* __restrict__ new_scores, int k, uint32_t* __restrict__ sorted_keys) {
   extern __shared__ __align__(16) uint32_t keys[];
   const int kpad = (k + 127) & ~127;
+#pragma unroll 8
   for (int t = threadIdx.x; t < kpad; t += kSortThreads)
-    keys[t] = t < k ? key_of_bits(canonical_bits(new_scores[t])) : 0xFFFFFFFFu;
+    keys[t] = t < k ? key_of_bits(canonical_bits(__ldg(new_scores + t))) : 0xFFFFFFFFu;
   __syncthreads();
   const int warps = kSortThreads / 32;
   const int lane = threadIdx.x & 31;
-  for (int j = blockIdx.x * warps + (threadIdx.x >> 5); j < k; j += gridDim.x * warps) {
-    const uint32_t kj = keys[j];
-    int lt = 0, le = 0;
+  for (int j0 = (blockIdx.x * warps + (threadIdx.x >> 5)) * 4; j0 < k; j0 += gridDim.x * warps * 4) {
+    const uint4 mine = *reinterpret_cast<const uint4*>(keys + j0);   // keys j0 .. j0 + 3 (padding beyond k)
+    const uint32_t kj[4] = {mine.x, mine.y, mine.z, mine.w};
+    int cnt[4] = {0, 0, 0, 0};
     for (int i = lane * 4; i < kpad; i += 128) {
       const uint4 q = *reinterpret_cast<const uint4*>(keys + i);
-      lt += (q.x < kj) + (q.y < kj) + (q.z < kj) + (q.w < kj);
-      le += (q.x <= kj) + (q.y <= kj) + (q.z <= kj) + (q.w <= kj);
+      if (i != j0) {
+        const uint32_t earlier = i < j0 ? 1u : 0u;   // canonical keys stay below 0xFFC00001: no overflow
+#pragma unroll
+        for (int y = 0; y < 4; ++y) {
+          const uint32_t t = kj[y] + earlier;
+          cnt[y] += (q.x < t) + (q.y < t) + (q.z < t) + (q.w < t);
+        }
+      } else {
+        const uint32_t qv[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int y = 0; y < 4; ++y)
+#pragma unroll
+          for (int x = 0; x < 4; ++x) cnt[y] += qv[x] < kj[y] + (x < y ? 1u : 0u);
+      }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      lt += __shfl_xor_sync(0xFFFFFFFFu, lt, o);
-      le += __shfl_xor_sync(0xFFFFFFFFu, le, o);
-    }
-    int slot = lt;
-    if (le - lt > 1) {  // equal keys: input order decides
-      int before = 0;
-      for (int i = lane; i < j; i += 32) before += keys[i] == kj;
+    for (int o = 16; o > 0; o >>= 1)
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, o);
-      slot += before;
+      for (int y = 0; y < 4; ++y) cnt[y] += __shfl_xor_sync(0xFFFFFFFFu, cnt[y], o);
+    if (lane < 4 && j0 + lane < k) {
+      const int slot = lane == 0 ? cnt[0] : lane == 1 ? cnt[1] : lane == 2 ? cnt[2] : cnt[3];
+      sorted_keys[slot] = keys[j0 + lane];
     }
-    if (lane == 0) sorted_keys[slot] = kj;
   }
 }
 
@@ -688,7 +697,8 @@ __global__ void __launch_bounds__(kMergeThreads)
 merge_kernel(const float* __restrict__ old_buf, int n, const uint32_t* __restrict__ new_keys, int k,
              float* __restrict__ out) {
   extern __shared__ uint32_t nk[];
-  for (int t = threadIdx.x; t < k; t += kMergeThreads) nk[t] = new_keys[t];
+#pragma unroll 8
+  for (int t = threadIdx.x; t < k; t += kMergeThreads) nk[t] = __ldg(new_keys + t);
   __syncthreads();
   // New keys first, one warp each: a 32-way search of the old buffer (every lane probes one of 32 evenly spaced
   // entries, a ballot keeps the interval between the last "<=" and the first ">"), so the chain of dependent
@@ -1042,6 +1052,7 @@ small_update_kernel(float* calib, int n, const float* __restrict__ new_scores, i
   uint32_t* ok = sm + k2;   // [n] keys of the old buffer
   for (int t = threadIdx.x; t < k2; t += kSmallUpdThreads)
     nk[t] = t < k ? key_of_bits(canonical_bits(new_scores[t])) : 0xFFFFFFFFu;
+#pragma unroll 8
   for (int t = threadIdx.x; t < n; t += kSmallUpdThreads) ok[t] = key_of_bits(canonical_bits(calib[t]));
   __syncthreads();
   for (int size = 2; size <= k2; size <<= 1) {
