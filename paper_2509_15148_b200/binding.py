@@ -43,11 +43,9 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
         return _lib
     path = _build.LIB_PATH
     if rebuild_if_stale and _build.is_stale():
-        try:
-            _build.build_library()
-        except Exception:
-            if not os.path.exists(path):
-                raise
+        # A library older than its sources is never loaded: if it cannot be rebuilt (no nvcc, or the sources no
+        # longer compile) this raises, so that nothing runs on a binary that does not match the tree.
+        _build.build_library()
     if not os.path.exists(path):
         raise RuntimeError(f"{path} is missing: build it with `python -m paper_2509_15148_b200.build`")
     lib = ctypes.CDLL(path)
