@@ -8,7 +8,9 @@ calibration buffer starting at n = 4096, alpha = 0.1):
     atts_score_logprob -> atts_conformal_rank -> atts_classify -> atts_calib_update
 
 The metric is draft tokens scored per second over the whole job.  `python bench.py --gpus N
---steps K --warmup W` (under torchrun for N > 1, one rank per GPU) prints one JSON line on rank 0.
+--steps K --warmup W` prints one JSON line on rank 0.  For N > 1 it runs one rank per GPU: started
+plainly it launches the N ranks itself (torch.distributed.run, loopback rendezvous); started under
+torchrun it is one of them.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
@@ -711,6 +713,15 @@ def main():
                     help="run only the conformal-only workload section and print it (for profiling those kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from paper_2509_15148_b200 import sharding
+    if sharding.needs_launch(args.gpus, os.environ):
+        # started as a plain `python bench.py --gpus N`: start the N ranks (one per GPU) and hand over to them
+        cmd, env = sharding.launch_command(os.path.abspath(__file__), sys.argv[1:], args.gpus, sharding.free_port(),
+                                           sys.executable, os.environ)
+        sys.exit(subprocess.run(cmd, env=env).returncode)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -8,6 +8,34 @@ buffers stay bit-identical without any further traffic.
 from __future__ import annotations
 
 
+def free_port() -> int:
+    """A TCP port that is free on the loopback interface right now."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_command(script: str, script_args: list[str], n_ranks: int, port: int, python: str,
+                   environ: dict) -> tuple[list[str], dict]:
+    """Command line and environment that start `script` as n_ranks processes on this node, one per GPU, with a
+    loopback rendezvous (torch.distributed.run).  NCCL's communicator lines are switched on unless the caller has
+    set NCCL_DEBUG already, so that the number of ranks of the communicator can be read from the log."""
+    if n_ranks < 2:
+        raise ValueError("one rank needs no launcher")
+    cmd = [python, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), script] + list(script_args)
+    env = dict(environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    return cmd, env
+
+
+def needs_launch(n_ranks: int, environ: dict) -> bool:
+    """True when more than one rank is asked for and this process was not started by a launcher already."""
+    return n_ranks > 1 and "WORLD_SIZE" not in environ
+
+
 def sample_range(n_samples: int, world: int, rank: int) -> tuple[int, int]:
     """Contiguous block [begin, end) of a batch of n_samples that `rank` scores (sizes differ by at most 1)."""
     if not (0 <= rank < world):

@@ -25,6 +25,20 @@ def test_reference_arm_prints_the_contract_keys():
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
 
 
+def test_plain_command_with_two_gpus_starts_two_ranks():
+    """`python bench.py --gpus 2` without a launcher starts two ranks itself; in the reference arm rank 0 alone works
+    and prints, the other rank exits 0 (this arm needs no GPU, so the launch path is exercised on CPU)."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--steps", "1", "--warmup", "0", "--oracle-rows", "8"], capture_output=True, text=True,
+                         timeout=900, cwd=ROOT, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [ln for ln in out.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+
+
 import pytest  # noqa: E402
 
 

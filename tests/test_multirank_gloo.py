@@ -107,3 +107,26 @@ def test_two_ranks_vocabulary_sharded_scoring(tmp_path):
     want = orc.token_logprob(inputs.hidden(1, 40, 32), inputs.lm_head(2, 700, 32), inputs.zipf_ids(3, 40, 700))
     for r in range(world):
         np.testing.assert_allclose(np.load(tmp_path / f"lp_{r}.npy"), want, atol=1e-12)
+
+
+def test_launcher_host_logic():
+    """`bench.py --gpus N` started plainly starts its own N ranks; under a launcher, or with one GPU, it does not."""
+    assert not sharding.needs_launch(1, {})
+    assert sharding.needs_launch(2, {})
+    assert not sharding.needs_launch(2, {"WORLD_SIZE": "2", "RANK": "0"})
+    cmd, env = sharding.launch_command("/x/bench.py", ["--gpus", "2", "--steps", "5"], 2, 29517, "/usr/bin/python",
+                                       {"PATH": "/bin", "NCCL_DEBUG": "WARN"})
+    assert cmd[:3] == ["/usr/bin/python", "-m", "torch.distributed.run"]
+    assert "--nproc-per-node=2" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29517"
+    assert cmd[-5:] == ["/x/bench.py", "--gpus", "2", "--steps", "5"]
+    assert env["NCCL_DEBUG"] == "WARN" and env["PATH"] == "/bin"          # the caller's settings win
+    _, env2 = sharding.launch_command("/x/bench.py", [], 4, 1, "py", {})
+    assert env2["NCCL_DEBUG"] == "INFO"
+    try:
+        sharding.launch_command("/x/bench.py", [], 1, 1, "py", {})
+        raise AssertionError("one rank must not be launched")
+    except ValueError:
+        pass
+    port = sharding.free_port()
+    assert 1024 <= port < 65536
