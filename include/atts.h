@@ -51,7 +51,7 @@ typedef enum {
 #define ATTS_DEV_TOKEN_ID_RANGE 1u /* a token id was outside [0, V): that row's log-prob is NaN */
 #define ATTS_DEV_WAIT_EXPIRED 2u   /* a pipeline wait in the scoring kernel ran out; outputs invalid */
 #define ATTS_DEV_GROUP_ID_RANGE 4u /* a group id was outside [0, G): that candidate has numer 0 */
-#define ATTS_DEV_INDEX_STALE 8u    /* atts_rank_classify_indexed: the index was built for another n; no output written */
+#define ATTS_DEV_INDEX_STALE 8u    /* an indexed call was given an index that does not describe fill n; nothing written */
 
 /* Stage labels written by atts_classify (the three stages of the rejection-sampling pipeline,
  * Sec. 3.3): the highest stage a sample reaches in this turn. */
@@ -273,30 +273,47 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
  * those of Eq. p-value, byte for byte what atts_rank_classify writes).
  *
  * Ranking many candidates against a buffer too large for shared memory is bound by the divergent loads
- * of each candidate's search.  A small index kept beside the buffer - the last entry of every aligned group
- * of 8 entries, and the last entry of every group of 64 laid out as a search tree - lets a candidate finish
- * with two 32-byte loads.  The index describes one fill n of one buffer: rebuild it whenever the buffer
- * changes.  atts_calib_update_indexed does so in the pass that writes the merged buffer back, at no extra
- * launch; atts_calib_index_build does it for a buffer filled some other way.
+ * of each candidate's search.  An index kept beside the buffer - a copy of the buffer, the last entry of every
+ * aligned group of 8, 64, ... entries, and the coarsest of those levels laid out as a search tree - lets a
+ * candidate finish with one to four 32-byte loads (two up to n = 524,223, three up to 4,193,791).  The index
+ * holds all of this twice: an update reads the half that describes the present fill and writes the other half
+ * and the caller's buffer in one pass, so it needs no copy back, and it touches nothing that a rank of the fill
+ * it started from reads.  The calibration state of a caller that uses these calls is the buffer AND its index:
+ * both describe the same fill n.
  *
  *   atts_calib_index_bytes   host out *bytes: size of an index for buffers of up to `cap` entries,
- *                            0 <= cap <= 524,223 (else ATTS_ERR_SHAPE: use the calls without an index)
- *   index         dev  256-byte aligned, at least atts_calib_index_bytes(n) bytes (ATTS_ERR_WORKSPACE)
- *   calib_sorted  dev  as for atts_conformal_rank; atts_rank_classify_indexed also needs it 32-byte aligned
- *   atts_calib_update_indexed   arguments and result as atts_calib_update; afterwards `index` describes
- *                            calib[0, n + k)
+ *                            0 <= cap < 2^24 - 1 (about 9.2 bytes per entry plus 64 KB)
+ *   index         dev  256-byte aligned; index_bytes: the size of that allocation, the same value in every call
+ *                      (the layout is derived from it); too small for n (+ k): ATTS_ERR_WORKSPACE
+ *   atts_calib_index_build   makes `index` describe calib_sorted[0, n) (a buffer filled some other way, or the
+ *                            start of a sequence)
+ *   atts_calib_update_indexed   arguments and result as atts_calib_update; `index` must describe calib[0, n)
+ *                            when the call runs and describes calib[0, n + k) afterwards, and it still holds
+ *                            the description of fill n until the next update.  If it does not describe fill n,
+ *                            nothing is changed and ATTS_DEV_INDEX_STALE is recorded.  (Small updates -
+ *                            n <= 28,672, k <= 4096, 8 k <= n + 64 - and k == 0 rebuild the index from the
+ *                            buffer instead and need no valid index.)
  *   atts_rank_classify_indexed  arguments and outputs as atts_rank_classify, but n_alpha may be 0 (rank and
- *                            p-values only; stage and stage_counts are then ignored).  If `index` was built
- *                            for another n nothing is written and ATTS_DEV_INDEX_STALE is recorded
- *                            (atts_last_device_status then returns ATTS_ERR_INDEX).
+ *                            p-values only; stage and stage_counts are then ignored).  With n > 8191 and
+ *                            Nc >= 16384 the candidates are ranked against the index's own copy of the buffer
+ *                            (calib_sorted is not read).  If `index` does not describe fill n nothing is written
+ *                            and ATTS_DEV_INDEX_STALE is recorded (atts_last_device_status then returns
+ *                            ATTS_ERR_INDEX).
+ *                            With stage_counts the call gathers the counts in a few words of the index header
+ *                            (which is why `index` is not const): two such calls on one index must not overlap.
+ * Overlap: atts_rank_classify_indexed for fill n and the atts_calib_update_indexed that starts from fill n may run
+ * at the same time (different streams).  The update after that one overwrites what that rank reads: order it
+ * behind the rank.
+ * Both kernels are launched with programmatic stream serialisation: they may be set up on the SMs while the kernel
+ * before them in the stream drains, and wait for its completion before they read anything.
  */
 int atts_calib_index_bytes(int64_t cap, size_t* bytes);
 int atts_calib_index_build(const float* calib_sorted, int64_t n, void* index, size_t index_bytes, void* cuda_stream);
-int atts_calib_update_indexed(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k,
-                              int64_t* n_out, void* index, size_t index_bytes, void* workspace,
-                              size_t workspace_bytes, void* cuda_stream);
+int atts_calib_update_indexed(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
+                              void* index, size_t index_bytes, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream);
 int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
-                               const void* index, const double* alphas, int32_t n_alpha, uint32_t* numer,
+                               void* index, const double* alphas, int32_t n_alpha, uint32_t* numer,
                                float* pvalue, uint8_t* stage, uint32_t* stage_counts, void* cuda_stream);
 
 /*
@@ -328,7 +345,7 @@ int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* cal
  */
 #define ATTS_STATIC_MAX_TOTAL 65536
 #define ATTS_STATIC_MAX_NEW 16384
-#define ATTS_STATIC_SCRATCH_BYTES (4 * ATTS_STATIC_MAX_NEW + 4 * ATTS_STATIC_MAX_TOTAL)
+#define ATTS_STATIC_SCRATCH_BYTES (4 * ATTS_STATIC_MAX_TOTAL)
 int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k,
                              int64_t* n_out, void* cuda_stream);
 

@@ -92,12 +92,11 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(sort_new_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      kSortMaxK * 4) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(small_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       4 * (kSmallUpdMaxOld + kSmallUpdMaxNew)) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      kSortMaxK * 4) == cudaSuccess;
+      const int merge_smem = 4 * (2 * kSortMaxK + kMergeTileMax);
+      ok = ok && cudaFuncSetAttribute(merge_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, merge_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(merge_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, merge_smem) == cudaSuccess;
       if (!ok) {
         cudaGetLastError();
         di.status = ATTS_ERR_CUDA;
@@ -115,6 +114,27 @@ struct Profile {
   cudaEvent_t* ev = nullptr;  // 2 * cap events
 };
 static Profile g_prof;
+
+// Launch with the programmatic-serialisation attribute: the kernel may be set up while its predecessor in the
+// stream drains; it calls pdl_wait() before it reads anything (see conformal.cuh).
+template <typename... KArgs, typename... Args>
+static int launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  return ATTS_OK;
+}
 
 static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 static inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -168,8 +188,7 @@ static int encode_2d(const DeviceInfo* di, CUtensorMap* map, const void* base, i
   return r == CUDA_SUCCESS ? ATTS_OK : ATTS_ERR_CUDA;
 }
 
-// Built-in scratch of atts_calib_update_static: [sorted new keys: ATTS_STATIC_MAX_NEW u32]
-// [merged copy: ATTS_STATIC_MAX_TOTAL f32].  In host code this name is only a handle for
+// Built-in scratch of atts_calib_update_static: the merged copy, ATTS_STATIC_MAX_TOTAL f32.  In host code this name is only a handle for
 // cudaGetSymbolAddress; the device address it yields is what kernels are given.
 static __device__ __align__(256) unsigned char g_static_scratch[ATTS_STATIC_SCRATCH_BYTES];
 static unsigned char* g_static_scratch_addr[64] = {};
@@ -382,6 +401,15 @@ int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float
 }
 
 // Shared launcher of the rank kernel, with or without the fused thresholding.
+static int zero_counts(uint32_t* counts, int n_alpha, cudaStream_t stream) {
+  if (counts && cudaMemsetAsync(counts, 0, (size_t)n_alpha * 3 * sizeof(uint32_t), stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  return ATTS_OK;
+}
+
+// A grid of one block stores its stage counts; larger grids add to counts the host has zeroed.
 static int launch_rank(const DeviceInfo* di, const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
                        uint32_t* numer, float* pvalue, int n_alpha, const FusedClassify& fc, cudaStream_t stream) {
   // Many candidates against a buffer that fits in shared memory: the bucket form (one table lookup and three
@@ -392,6 +420,7 @@ static int launch_rank(const DeviceInfo* di, const float* scores, int64_t Nc, co
     const int64_t per_blk = (int64_t)kRankThreads * kRankPerThread;
     int64_t nblk = (Nc + per_blk - 1) / per_blk;
     if (nblk > di->sm_count) nblk = di->sm_count;
+    if (nblk > 1 && n_alpha > 0 && zero_counts(fc.counts, n_alpha, stream) != ATTS_OK) return ATTS_ERR_CUDA;
     const dim3 g((unsigned)nblk), b(kRankThreads);
     const size_t sm = 4 * (((size_t)1 << Blog2) + 1 + (size_t)n + kBucketPad + (pvalue ? (size_t)n + 2 : 0));
     switch (n_alpha) {
@@ -417,6 +446,7 @@ static int launch_rank(const DeviceInfo* di, const float* scores, int64_t Nc, co
   // one block per SM when the table is filled by strided loads (the fill is paid per block), two otherwise
   const int64_t max_blocks = (int64_t)di->sm_count * (L == 0 ? 2 : 1);
   if (blocks > max_blocks) blocks = max_blocks;
+  if (blocks > 1 && n_alpha > 0 && zero_counts(fc.counts, n_alpha, stream) != ATTS_OK) return ATTS_ERR_CUDA;
   const dim3 grid((unsigned)blocks), block(kRankThreads);
   const size_t smem = ((size_t)4 << P) + (L == 0 ? (size_t)4 * (n + 2) : 0);  // table (+ p-value table)
   switch (n_alpha) {
@@ -459,11 +489,7 @@ int atts_rank_classify(const float* scores, int64_t Nc, const float* calib_sorte
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (stage_counts && cudaMemsetAsync(stage_counts, 0, (size_t)n_alpha * 3 * sizeof(uint32_t), stream) != cudaSuccess) {
-    cudaGetLastError();
-    return ATTS_ERR_CUDA;
-  }
-  if (Nc == 0) return ATTS_OK;
+  if (Nc == 0) return zero_counts(stage_counts, n_alpha, stream);
   FusedClassify fc{};
   for (int a = 0; a < n_alpha; ++a) {
     fc.k_alpha[a] = (uint32_t)floor(alphas[a] * (double)(n + 1));
@@ -483,16 +509,13 @@ int atts_classify(const uint32_t* numer, int64_t Nc, int64_t n, double alpha, ui
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (stage_counts && cudaMemsetAsync(stage_counts, 0, 3 * sizeof(uint32_t), stream) != cudaSuccess) {
-    cudaGetLastError();
-    return ATTS_ERR_CUDA;
-  }
-  if (Nc == 0) return ATTS_OK;
+  if (Nc == 0) return zero_counts(stage_counts, 1, stream);
   const uint32_t k_alpha = (uint32_t)floor(alpha * (double)(n + 1));
   const int64_t per_block = (int64_t)kClassifyThreads * kClassifyPerThread;
   int64_t blocks = (Nc + per_block - 1) / per_block;
   const int64_t max_blocks = (int64_t)di->sm_count * 8;
   if (blocks > max_blocks) blocks = max_blocks;
+  if (blocks > 1 && zero_counts(stage_counts, 1, stream) != ATTS_OK) return ATTS_ERR_CUDA;   // one block stores its counts
   classify_kernel<<<(unsigned)blocks, kClassifyThreads, 0, stream>>>(numer, Nc, k_alpha, stage, stage_counts);
   return launch_status();
 }
@@ -519,23 +542,21 @@ int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, u
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (stage_counts && cudaMemsetAsync(stage_counts, 0, 3 * sizeof(uint32_t), stream) != cudaSuccess) {
-    cudaGetLastError();
-    return ATTS_ERR_CUDA;
-  }
-  if (Nc == 0) return ATTS_OK;
+  if (Nc == 0) return zero_counts(stage_counts, 1, stream);
   const int64_t per_block = (int64_t)kClassifyThreads * kClassifyPerThread;
   int64_t blocks = (Nc + per_block - 1) / per_block;
   const int64_t max_blocks = (int64_t)di->sm_count * 8;
   if (blocks > max_blocks) blocks = max_blocks;
+  if (blocks > 1 && zero_counts(stage_counts, 1, stream) != ATTS_OK) return ATTS_ERR_CUDA;   // one block stores its counts
   classify_threshold_kernel<<<(unsigned)blocks, kClassifyThreads, 0, stream>>>(scores, Nc, tau, stage, stage_counts);
   return launch_status();
 }
 
+// Workspace of atts_takeover_ids: [one 64-bit word per tile][ticket counter], cleared before the launch.
 int atts_takeover_ids_workspace_bytes(int64_t Nc, size_t* bytes) {
   if (!bytes) return ATTS_ERR_NULL;
   if (Nc < 0 || Nc >= (1ll << 31)) return ATTS_ERR_SHAPE;
-  *bytes = round_up((size_t)((Nc + kIdsTile - 1) / kIdsTile) * sizeof(uint32_t), 256) + 256;
+  *bytes = round_up((size_t)((Nc + kIdsTile - 1) / kIdsTile) * sizeof(unsigned long long) + 8, 256) + 256;
   return ATTS_OK;
 }
 
@@ -560,12 +581,15 @@ int atts_takeover_ids(const uint8_t* stage, int64_t Nc, int32_t* ids, int64_t id
   }
   const int tiles = (int)((Nc + kIdsTile - 1) / kIdsTile);
   const bool vec = aligned(stage, 16);
-  uint32_t* tile_count = static_cast<uint32_t*>(workspace);
-  takeover_count_kernel<<<tiles, kIdsThreads, 0, stream>>>(stage, Nc, vec, tile_count);
-  if ((st = launch_status()) != ATTS_OK) return st;
-  takeover_scan_kernel<<<1, kIdsThreads, 0, stream>>>(tile_count, tiles, count);
-  if ((st = launch_status()) != ATTS_OK) return st;
-  takeover_write_kernel<<<tiles, kIdsThreads, 0, stream>>>(stage, Nc, vec, tile_count, ids, ids_cap);
+  unsigned long long* state = static_cast<unsigned long long*>(workspace);
+  unsigned int* ticket = reinterpret_cast<unsigned int*>(state + tiles);
+  if (tiles > 1 && cudaMemsetAsync(workspace, 0, (size_t)tiles * sizeof(unsigned long long) + 8, stream) != cudaSuccess) {
+    cudaGetLastError();
+    return ATTS_ERR_CUDA;
+  }
+  int blocks = tiles < di->sm_count * 6 ? tiles : di->sm_count * 6;
+  takeover_ids_kernel<<<blocks, kIdsThreads, 0, stream>>>(stage, Nc, tiles, vec, state, ticket, ids, ids_cap, count,
+                                                         di->dev_status);
   return launch_status();
 }
 
@@ -612,40 +636,53 @@ int atts_classify_conditional(const uint32_t* numer, const uint32_t* denom, int6
 }
 
 // ---- calibration index (see rank_indexed_kernel) ----
-static inline int index_levels(int64_t n, int* ns_out) {
-  const int ns = (int)(n / 64) + 1;
-  int P = 1;
-  while ((1 << P) - 1 < ns) ++P;
-  *ns_out = ns;
-  return P;
-}
-static inline size_t index_bytes_for(int64_t n) {
-  return 4 * ((size_t)kIndexHeaderWords + kIndexTreeWords + 8 * ((size_t)(n / 64) + 1));
+static inline size_t index_bytes_for(int64_t cap) { return 4 * index_words((uint32_t)cap); }
+
+// The capacity an index of `index_bytes` bytes is laid out for: the largest one that fits.  Every call that is
+// given the same allocation therefore agrees on the layout.
+static int64_t index_cap_of_bytes(size_t index_bytes) {
+  if (index_bytes < index_bytes_for(0)) return -1;
+  int64_t lo = 0, hi = (1ll << 24) - 2;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi + 1) / 2;
+    if (index_bytes_for(mid) <= index_bytes) lo = mid; else hi = mid - 1;
+  }
+  return lo;
 }
 
-// Launches the index build for src[0, n); copy_to != nullptr: also copies src to copy_to.
-static int launch_index_build(const DeviceInfo* di, const float* src, float* copy_to, int64_t n, void* index,
+// Launches the build of slot 0 of the index from src[0, n).
+static int launch_index_build(const DeviceInfo* di, const float* src, int64_t n, void* index, int64_t index_cap,
                               cudaStream_t stream) {
-  int ns = 0;
-  const int P = index_levels(n, &ns);
-  int64_t work = n > (1ll << P) ? n : (1ll << P);
-  if (work < 8 * (int64_t)ns) work = 8 * (int64_t)ns;
+  int64_t work = n > 8192 ? n : 8192;
   int64_t blocks = (work + 255) / 256;
   if (blocks > (int64_t)di->sm_count * 8) blocks = (int64_t)di->sm_count * 8;
-  if (copy_to)
-    index_build_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(src, copy_to, (int)n, P, ns, static_cast<uint32_t*>(index));
-  else
-    index_build_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(src, nullptr, (int)n, P, ns, static_cast<uint32_t*>(index));
+  index_build_kernel<<<(unsigned)blocks, 256, 0, stream>>>(src, (int)n, (uint32_t)index_cap, static_cast<uint32_t*>(index));
   return launch_status();
 }
 
-// Workspace of atts_calib_update: [sorted new keys: min(k, kSortMaxK) u32][merged copy: n + k f32]
+// Workspace of atts_calib_update: the merged copy, n + k f32.
 int atts_calib_workspace_bytes(int64_t n, int64_t k, size_t* bytes) {
   if (!bytes) return ATTS_ERR_NULL;
   if (n < 0 || k < 0 || n + k >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
-  const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
-  *bytes = round_up((size_t)kk * 4, 256) + round_up((size_t)(n + k) * 4, 256) + 256;
+  *bytes = round_up((size_t)(n + k) * 4, 256) + 256;
   return ATTS_OK;
+}
+
+// One launch of the merge kernel: kc <= kSortMaxK new scores into cur old entries.  index != nullptr: from the index
+// slot of fill `cur` into the other slot and `out` (the caller's buffer); else from calib into `out` (scratch).
+static int launch_merge(const DeviceInfo* di, const float* calib, int64_t cur, const float* new_scores, int kc, float* out,
+                        void* index, int64_t index_cap, cudaStream_t stream) {
+  int k2 = kMergeThreads;   // the block's sort pads its keys to a multiple of the block size
+  while (k2 < kc) k2 <<= 1;
+  int tile_len = 0, tiles = 0;
+  merge_tiling((int)cur, di->sm_count, tile_len, tiles);
+  const int blocks = tiles < di->sm_count ? tiles : di->sm_count;
+  const size_t smem = (size_t)4 * (2 * (size_t)k2 + (size_t)tile_len);
+  if (index)
+    return launch_pdl(merge_kernel<true>, dim3(blocks), dim3(kMergeThreads), smem, stream, nullptr, (int)cur, new_scores, kc, k2,
+                      tile_len, tiles, out, static_cast<uint32_t*>(index), (uint32_t)index_cap, di->dev_status);
+  return launch_pdl(merge_kernel<false>, dim3(blocks), dim3(kMergeThreads), smem, stream, calib, (int)cur, new_scores, kc, k2,
+                    tile_len, tiles, out, nullptr, 0u, di->dev_status);
 }
 
 static int calib_update_impl(float* calib, int64_t n, int64_t cap, const float* new_scores, int64_t k, int64_t* n_out,
@@ -660,43 +697,33 @@ static int calib_update_impl(float* calib, int64_t n, int64_t cap, const float* 
   const DeviceInfo* di;
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
+  int64_t index_cap = 0;
   if (index) {
-    if (n + k > kIndexMaxN) return ATTS_ERR_SHAPE;
     if (!aligned(index, 256)) return ATTS_ERR_ALIGN;
-    if (index_bytes < index_bytes_for(n + k)) return ATTS_ERR_WORKSPACE;
+    index_cap = index_cap_of_bytes(index_bytes);
+    if (index_cap < n + k) return ATTS_ERR_WORKSPACE;
   }
   if (n_out) *n_out = n + k;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (k == 0) return index ? launch_index_build(di, calib, nullptr, n, index, stream) : ATTS_OK;
-  const int64_t kk = k < kSortMaxK ? k : kSortMaxK;
-  uint32_t* sorted_keys = static_cast<uint32_t*>(workspace);
-  float* merged = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + round_up((size_t)kk * 4, 256));
+  if (k == 0) return index ? launch_index_build(di, calib, n, index, index_cap, stream) : ATTS_OK;
   // Small problems: one block does it in place in one launch.
   if (n <= kSmallUpdMaxOld && k <= kSmallUpdMaxNew && k * 8 <= n + 64) {
     int k2 = 1;
     while (k2 < k) k2 <<= 1;
     small_update_kernel<<<1, kSmallUpdThreads, (size_t)4 * (k2 + n), stream>>>(calib, (int)n, new_scores, (int)k, k2);
     if ((st = launch_status()) != ATTS_OK) return st;
-    return index ? launch_index_build(di, calib, nullptr, n + k, index, stream) : ATTS_OK;
+    return index ? launch_index_build(di, calib, n + k, index, index_cap, stream) : ATTS_OK;
   }
-  // Sort the new keys, merge into the workspace, copy back.  Batches larger than one sort launch handles are
-  // inserted slice by slice.
+  // One merge launch per slice of at most kSortMaxK new scores: with an index, from one slot of the index into the
+  // other and the buffer itself; without, into the workspace followed by a copy back.
+  float* merged = static_cast<float*>(workspace);
   int64_t cur = n;
   for (int64_t off = 0; off < k; off += kSortMaxK) {
     const int kc = (int)((k - off) < kSortMaxK ? (k - off) : kSortMaxK);
-    int sort_blocks = (kc + kSortKeysPerBlock - 1) / kSortKeysPerBlock;
-    if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
-    sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)((kc + 127) & ~127) * 4, stream>>>(new_scores + off, kc, sorted_keys);
-    if ((st = launch_status()) != ATTS_OK) return st;
-    int64_t total = cur + kc;
-    int merge_blocks = (int)((total + kMergeThreads - 1) / kMergeThreads);
-    if (merge_blocks > di->sm_count * 4) merge_blocks = di->sm_count * 4;
-    merge_kernel<<<merge_blocks, kMergeThreads, (size_t)kc * 4, stream>>>(calib, (int)cur, sorted_keys, kc, merged);
-    if ((st = launch_status()) != ATTS_OK) return st;
-    if (index && off + kSortMaxK >= k) {
-      // last slice: the copy back also writes the index of the merged buffer
-      if ((st = launch_index_build(di, merged, calib, total, index, stream)) != ATTS_OK) return st;
-    } else if (cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+    const int64_t total = cur + kc;
+    if ((st = launch_merge(di, calib, cur, new_scores + off, kc, index ? calib : merged, index, index_cap, stream)) != ATTS_OK)
+      return st;
+    if (!index && cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
       cudaGetLastError();
       return ATTS_ERR_CUDA;
     }
@@ -732,19 +759,9 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
   if (n_out) *n_out = n + k;
   if (k == 0) return ATTS_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  uint32_t* sorted_keys = reinterpret_cast<uint32_t*>(scratch);
-  float* merged = reinterpret_cast<float*>(scratch + 4 * ATTS_STATIC_MAX_NEW);
-  const int kc = (int)k;
-  int sort_blocks = (kc + kSortKeysPerBlock - 1) / kSortKeysPerBlock;
-  if (sort_blocks > di->sm_count * 8) sort_blocks = di->sm_count * 8;
-  sort_new_kernel<<<sort_blocks, kSortThreads, (size_t)((kc + 127) & ~127) * 4, stream>>>(new_scores, kc, sorted_keys);
-  if ((st = launch_status()) != ATTS_OK) return st;
-  const int64_t total = n + k;
-  int merge_blocks = (int)((total + kMergeThreads - 1) / kMergeThreads);
-  if (merge_blocks > di->sm_count * 4) merge_blocks = di->sm_count * 4;
-  merge_kernel<<<merge_blocks, kMergeThreads, (size_t)kc * 4, stream>>>(calib, (int)n, sorted_keys, kc, merged);
-  if ((st = launch_status()) != ATTS_OK) return st;
-  if (cudaMemcpyAsync(calib, merged, (size_t)total * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
+  float* merged = reinterpret_cast<float*>(scratch);
+  if ((st = launch_merge(di, calib, n, new_scores, (int)k, merged, nullptr, 0, stream)) != ATTS_OK) return st;
+  if (cudaMemcpyAsync(calib, merged, (size_t)(n + k) * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess) {
     cudaGetLastError();
     return ATTS_ERR_CUDA;
   }
@@ -753,45 +770,41 @@ int atts_calib_update_static(float* calib, int64_t n, int64_t cap, const float* 
 
 int atts_calib_index_bytes(int64_t cap, size_t* bytes) {
   if (!bytes) return ATTS_ERR_NULL;
-  if (cap < 0 || cap > kIndexMaxN) return ATTS_ERR_SHAPE;
+  if (cap < 0 || cap >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
   *bytes = round_up(index_bytes_for(cap), 256);
   return ATTS_OK;
 }
 
 int atts_calib_index_build(const float* calib_sorted, int64_t n, void* index, size_t index_bytes, void* cuda_stream) {
-  if (n < 0 || n > kIndexMaxN) return ATTS_ERR_SHAPE;
+  if (n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
   if (!index || (n > 0 && !calib_sorted)) return ATTS_ERR_NULL;
   if (!aligned(calib_sorted, 4) || !aligned(index, 256)) return ATTS_ERR_ALIGN;
-  if (index_bytes < index_bytes_for(n)) return ATTS_ERR_WORKSPACE;
+  const int64_t index_cap = index_cap_of_bytes(index_bytes);
+  if (index_cap < n) return ATTS_ERR_WORKSPACE;
   const DeviceInfo* di;
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
-  return launch_index_build(di, calib_sorted, nullptr, n, index, static_cast<cudaStream_t>(cuda_stream));
+  return launch_index_build(di, calib_sorted, n, index, index_cap, static_cast<cudaStream_t>(cuda_stream));
 }
 
-int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n, const void* index,
+int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n, void* index,
                                const double* alphas, int32_t n_alpha, uint32_t* numer, float* pvalue, uint8_t* stage,
                                uint32_t* stage_counts, void* cuda_stream) {
-  if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n > kIndexMaxN) return ATTS_ERR_SHAPE;
+  if (Nc < 0 || Nc >= (1ll << 31) || n < 0 || n >= (1ll << 24) - 1) return ATTS_ERR_SHAPE;
   if (n_alpha < 0 || n_alpha > kMaxAlphas) return ATTS_ERR_ARG;
   if (n_alpha > 0 && !alphas) return ATTS_ERR_NULL;
   for (int a = 0; a < n_alpha; ++a)
     if (!(alphas[a] > 0.0 && alphas[a] < 1.0)) return ATTS_ERR_ARG;
   if (!index || (Nc > 0 && (!scores || !numer || (n_alpha > 0 && !stage)))) return ATTS_ERR_NULL;
   if (n > 0 && !calib_sorted) return ATTS_ERR_NULL;
-  if (!aligned(scores, 16) || !aligned(numer, 16) || !aligned(pvalue, 16) || !aligned(calib_sorted, 32) ||
+  if (!aligned(scores, 16) || !aligned(numer, 16) || !aligned(pvalue, 16) || !aligned(calib_sorted, 4) ||
       !aligned(index, 256) || !aligned(stage, 16) || !aligned(stage_counts, 4) || (n_alpha > 1 && Nc % 16 != 0))
     return ATTS_ERR_ALIGN;
   const DeviceInfo* di;
   int st = device_info(&di);
   if (st != ATTS_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (n_alpha > 0 && stage_counts &&
-      cudaMemsetAsync(stage_counts, 0, (size_t)n_alpha * 3 * sizeof(uint32_t), stream) != cudaSuccess) {
-    cudaGetLastError();
-    return ATTS_ERR_CUDA;
-  }
-  if (Nc == 0) return ATTS_OK;
+  if (Nc == 0) return zero_counts(stage_counts, n_alpha, stream);
   FusedClassify fc{};
   for (int a = 0; a < n_alpha; ++a) {
     fc.k_alpha[a] = (uint32_t)floor(alphas[a] * (double)(n + 1));
@@ -801,22 +814,21 @@ int atts_rank_classify_indexed(const float* scores, int64_t Nc, const float* cal
   // A buffer that fits in shared memory, or few candidates, gain nothing from the index.
   if (n <= kBucketMaxN || Nc < kIndexMinCandidates)
     return launch_rank(di, scores, Nc, calib_sorted, n, numer, pvalue, n_alpha, fc, stream);
-  int ns = 0;
-  const int P = index_levels(n, &ns);
+  const IndexShape sh = index_shape(n);
   const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
   int64_t blocks = (Nc + per_block - 1) / per_block;
   if (blocks > di->sm_count) blocks = di->sm_count;
   const dim3 grid((unsigned)blocks), block(kRankThreads);
-  const size_t smem = (size_t)4 << P;
-  const uint32_t* ix = static_cast<const uint32_t*>(index);
+  const size_t smem = (size_t)4 << sh.P;
+  // The stage counts are gathered in the index header and moved to stage_counts by the last block: no memset node.
+  uint32_t* ix = static_cast<uint32_t*>(index);
   switch (n_alpha) {
-    case 0: rank_indexed_kernel<0><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
-    case 1: rank_indexed_kernel<1><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
-    case 2: rank_indexed_kernel<2><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
-    case 3: rank_indexed_kernel<3><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
-    default: rank_indexed_kernel<4><<<grid, block, smem, stream>>>(scores, Nc, calib_sorted, (int)n, P, ix, numer, pvalue, fc, di->dev_status); break;
+    case 0: return launch_pdl(rank_indexed_kernel<0>, grid, block, smem, stream, scores, Nc, (int)n, ix, numer, pvalue, fc, di->dev_status);
+    case 1: return launch_pdl(rank_indexed_kernel<1>, grid, block, smem, stream, scores, Nc, (int)n, ix, numer, pvalue, fc, di->dev_status);
+    case 2: return launch_pdl(rank_indexed_kernel<2>, grid, block, smem, stream, scores, Nc, (int)n, ix, numer, pvalue, fc, di->dev_status);
+    case 3: return launch_pdl(rank_indexed_kernel<3>, grid, block, smem, stream, scores, Nc, (int)n, ix, numer, pvalue, fc, di->dev_status);
+    default: return launch_pdl(rank_indexed_kernel<4>, grid, block, smem, stream, scores, Nc, (int)n, ix, numer, pvalue, fc, di->dev_status);
   }
-  return launch_status();
 }
 
 int atts_last_device_status(void* cuda_stream, uint32_t* bits) {

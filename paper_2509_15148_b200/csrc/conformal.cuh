@@ -6,6 +6,14 @@
 
 namespace atts {
 
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialisation attribute may be set up
+// on the SMs while the kernel before it in the stream is still running; pdl_wait() returns once that kernel has
+// completed and its writes are visible, so nothing another kernel may have produced is read before it.
+// pdl_launch_dependents() lets the kernel after this one be set up early in the same way.  Both are no-ops for a
+// kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------------------------------------
 // Ordering of scores.  Candidates are compared with calibration scores as floats (a tie counts,
 // -0 == +0).  The calibration buffer itself is ordered by a monotone 32-bit key of the
@@ -145,11 +153,13 @@ struct FusedClassify {
   uint32_t* counts;  // [NA][3] or nullptr
 };
 
-// Per-thread tallies of the fused thresholding, and the code both rank kernels share: writing the numerators,
+// Per-thread tallies of the fused thresholding, and the code the rank kernels share: writing the numerators,
 // p-values and stage bytes of four candidates, and the block's contribution to the stage counts.
+// Stage from the numerator with unsigned arithmetic: numer - 1 < k_alpha holds exactly for 1 <= numer <= k_alpha
+// (numer = 0 wraps to the largest value), so stage = 2 + [numer - 1 < k_alpha] - [numer == 0].
 template <int NA>
 struct StageTally {
-  uint32_t c1[NA > 0 ? NA : 1] = {}, c3[NA > 0 ? NA : 1] = {}, seen = 0;
+  uint32_t c3[NA > 0 ? NA : 1] = {}, c1 = 0, seen = 0;   // stage-1 samples (no score) are the same for every alpha
 };
 
 template <int NA>
@@ -168,14 +178,20 @@ __device__ __forceinline__ void emit_four(int64_t j, int64_t Nc, bool full, cons
   if (NA > 0) {
     const int valid = full ? 4 : (int)(Nc - j);
     tally.seen += (uint32_t)valid;
+    uint32_t none[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      none[e] = (r[e] == 0u) ? 1u : 0u;
+      tally.c1 += (e < valid) ? none[e] : 0u;
+    }
 #pragma unroll
     for (int a = 0; a < NA; ++a) {
       uint32_t st[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        st[e] = stage_of(r[e], fc.k_alpha[a]);
-        tally.c1[a] += (e < valid) && (st[e] == 1u);
-        tally.c3[a] += (e < valid) && (st[e] == 3u);
+        const uint32_t rej = (r[e] - 1u < fc.k_alpha[a]) ? 1u : 0u;
+        st[e] = 2u + rej - none[e];
+        tally.c3[a] += (e < valid) ? rej : 0u;
       }
       if (full) {
         *reinterpret_cast<uint32_t*>(fc.stage[a] + j) = st[0] | (st[1] << 8) | (st[2] << 16) | (st[3] << 24);
@@ -186,15 +202,19 @@ __device__ __forceinline__ void emit_four(int64_t j, int64_t Nc, bool full, cons
   }
 }
 
-// Adds the block's stage counts to fc.counts ([NA][3]); every thread of the block calls it.
+// The block's stage counts go to fc.counts ([NA][3]); every thread of the block calls it.  A grid of one block
+// stores them; a larger grid adds them either to fc.counts itself (zeroed by the host before the launch:
+// scratch == nullptr) or to 12 zeroed scratch words followed by a counter of finished blocks, in which case the
+// last block to finish moves the totals to fc.counts and leaves the scratch zeroed for the next launch.
 template <int NA>
-__device__ __forceinline__ void flush_tally(const FusedClassify& fc, const StageTally<NA>& tally) {
+__device__ __forceinline__ void flush_tally(const FusedClassify& fc, const StageTally<NA>& tally, uint32_t* scratch = nullptr) {
   if (NA == 0 || fc.counts == nullptr) return;
   __shared__ uint32_t sh[kMaxAlphas][3][kRankThreads / 32];
+  __shared__ bool last_block;
   const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
 #pragma unroll
   for (int a = 0; a < NA; ++a) {
-    uint32_t v1 = tally.c1[a], v3 = tally.c3[a], v2 = tally.seen - tally.c1[a] - tally.c3[a];
+    uint32_t v1 = tally.c1, v3 = tally.c3[a], v2 = tally.seen - tally.c1 - tally.c3[a];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       v1 += __shfl_xor_sync(0xFFFFFFFFu, v1, o);
@@ -204,12 +224,22 @@ __device__ __forceinline__ void flush_tally(const FusedClassify& fc, const Stage
     if (l == 0) { sh[a][0][w] = v1; sh[a][1][w] = v2; sh[a][2][w] = v3; }
   }
   __syncthreads();
+  uint32_t t = 0;
   if ((int)threadIdx.x < NA * 3) {
     const int a = threadIdx.x / 3, i = threadIdx.x % 3;
-    uint32_t t = 0;
     for (int q = 0; q < kRankThreads / 32; ++q) t += sh[a][i][q];
-    if (t) atomicAdd(fc.counts + threadIdx.x, t);
+    if (gridDim.x == 1) fc.counts[threadIdx.x] = t;
+    else if (t) atomicAdd((scratch ? scratch : fc.counts) + threadIdx.x, t);
   }
+  if (gridDim.x == 1 || scratch == nullptr) return;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last_block = atomicAdd(scratch + 3 * kMaxAlphas, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last_block) return;
+  __threadfence();
+  if ((int)threadIdx.x < NA * 3) fc.counts[threadIdx.x] = atomicExch(scratch + threadIdx.x, 0u);
+  if (threadIdx.x == 0) atomicExch(scratch + 3 * kMaxAlphas, 0u);
 }
 
 template <int NA>
@@ -430,21 +460,70 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
 // ---------------------------------------------------------------------------------------------
 // K3, indexed form: many candidates against a buffer too large for shared memory.
 //
-// The plain kernel pays, per block, one strided load for each of up to 8191 splitters, and per candidate up to
-// three dependent 4-byte loads plus one 32-byte load from the L2-resident buffer; divergent loads are served at
-// one per cycle per SM, so they are what bounds it.  An index kept beside the buffer (rebuilt whenever the
-// buffer changes, in the pass that writes the buffer anyway) removes most of them:
-//   aux[i]  = calib[8 i + 7], the last entry of every aligned group of 8 (NaN where that lies beyond n);
-//   tree    = the entries aux[8 r + 7] = calib[64 r + 63], r < ns = n / 64 + 1 (the last one always NaN), as an
-//             implicit search tree in breadth-first order, ready to be copied into shared memory row by row.
-// A candidate descends the tree (P shared-memory steps) to its group of 64, reads that group's 8 aux entries
-// in one 32-byte load to find its group of 8, and reads that group in a second 32-byte load.
-// Layout of the index (32-bit words): [0] n  [1] P  [2] ns  [3..7] 0  [8 ..) tree, kIndexTreeWords  [..) aux, 8 ns.
+// The plain kernel pays, per block, one strided load for each of up to 8191 splitters, and per candidate several
+// dependent loads from the L2-resident buffer; an SM serves divergent loads at one cache line per cycle, so they
+// are what bounds it.  A calibration index kept beside the buffer removes most of them.  It holds, twice (two
+// slots, see below):
+//   buf     a copy of the sorted buffer, 32-byte aligned;
+//   aux_a   a = 1 .. A: the last entry of every aligned group of 8^a entries, aux_a[i] = buf[8^a i + 8^a - 1]
+//           (NaN where that lies beyond n);
+//   tree    the last entries of the groups of G = 8^(A+1) entries, r < ns = n / G + 1 (the last one always NaN), as an
+//           implicit search tree in breadth-first order, ready to be copied into shared memory.
+// A candidate descends the tree (P shared-memory steps) to its group of G, then narrows by a factor of 8 per
+// 32-byte load: A loads of aux entries and one of the buffer.  A is the smallest number of levels for which the
+// tree has at most 8191 nodes: 0 for n < 65,528, 1 up to 524,223, 2 up to 4,193,791, 3 beyond.
+//
+// Two slots.  An update reads the buffer copy of the slot that describes the present fill n and writes the merged
+// buffer to the other slot and to the caller's buffer, together with the other slot's aux entries and tree: no
+// copy back, and nothing an update writes is read by a rank of the fill it started from, so the two may overlap.
+// A kernel finds its slot by the fill it is given: slot descriptors hold the fill they describe.
+//
+// Layout (32-bit words): header [64]: [0] magic [1] capacity the layout was made for
+//   [8 + 8 s ..] slot s: fill n (0xFFFFFFFF: none), P, A, ns;   [32 .. 45) zero between launches: scratch of the
+//   rank kernel's stage counts;   then slot 0, slot 1, each: tree [8192],
+//   aux_1, aux_2, aux_3, buf (every array a multiple of 8 words long).
 // ---------------------------------------------------------------------------------------------
-constexpr int kIndexHeaderWords = 8;
+constexpr int kIndexHeaderWords = 64;
 constexpr int kIndexTreeWords = 1 << kRankMaxTableLog2;               // 8191 nodes + 1 pad
-constexpr int64_t kIndexMaxN = 64ll * ((1 << kRankMaxTableLog2) - 1) - 1;   // ns = n / 64 + 1 <= 8191
+constexpr int kIndexMaxLevels = 3;
+constexpr int kIndexCountScratch = 32;   // header words [32, 45): stage-count accumulators of the rank kernel, block counter
+constexpr uint32_t kIndexMagic = 0x41545832u;
+constexpr uint32_t kIndexNoFill = 0xFFFFFFFFu;
 constexpr int64_t kIndexMinCandidates = 1 << 14;
+
+struct IndexLayout {
+  uint32_t aux_off[kIndexMaxLevels];   // word offsets inside a slot
+  uint32_t buf_off;
+  uint32_t slot_words;
+};
+__host__ __device__ inline IndexLayout index_layout(uint32_t cap) {
+  IndexLayout L;
+  uint32_t off = kIndexTreeWords;
+  for (int a = 0; a < kIndexMaxLevels; ++a) {
+    L.aux_off[a] = off;
+    off += ((cap >> (3 * (a + 1))) + 16u) & ~7u;   // entries up to 8 * (n >> 3(a+1)) + 7 are read
+  }
+  L.buf_off = off;
+  off += (cap + 15u) & ~7u;
+  L.slot_words = (off + 63u) & ~63u;
+  return L;
+}
+__host__ __device__ inline size_t index_words(uint32_t cap) {
+  return (size_t)kIndexHeaderWords + 2 * (size_t)index_layout(cap).slot_words;
+}
+// Shape of the index of a fill n: aux levels A, tree depth P, tree entries ns.
+struct IndexShape {
+  int A, P, ns;
+};
+__host__ __device__ inline IndexShape index_shape(int64_t n) {
+  IndexShape s;
+  s.A = 0;
+  while ((n >> (3 * (s.A + 1))) + 1 > (1 << kRankMaxTableLog2) - 1) ++s.A;
+  s.ns = (int)(n >> (3 * (s.A + 1))) + 1;
+  s.P = 1;
+  while ((1 << s.P) - 1 < s.ns) ++s.P;
+  return s;
+}
 
 // Slot, in the breadth-first table of a P-level tree, of the splitter with sorted rank r (inverse of the fill rule
 // of rank_kernel: node b at depth l holds rank (2q + 1) * 2^(P-1-l) - 1, q = b - 2^l).
@@ -455,57 +534,107 @@ __device__ __forceinline__ int index_slot_of_rank(int r, int P) {
   return (1 << depth) + (x >> (tz + 1)) - 1;
 }
 
-// Writes the index of src[0, n); with COPY also dst[e] = src[e] (the copy-back of a merge), so a calibration
-// update rebuilds the index in the pass that moves the merged buffer anyway.
-template <bool COPY>
-__global__ void __launch_bounds__(256)
-index_build_kernel(const float* __restrict__ src, float* __restrict__ dst, int n, int P, int ns,
-                   uint32_t* __restrict__ index) {
-  float* const tree = reinterpret_cast<float*>(index + kIndexHeaderWords);
-  float* const aux = tree + kIndexTreeWords;
-  const float qnan = __uint_as_float(0x7FC00000u);
-  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x;
-  if (tid < kIndexHeaderWords) index[tid] = tid == 0 ? (uint32_t)n : tid == 1 ? (uint32_t)P : tid == 2 ? (uint32_t)ns : 0u;
-  for (int e = tid; e < n; e += nthreads) {
-    const float v = src[e];
-    if (COPY) dst[e] = v;
-    if ((e & 7) == 7) aux[e >> 3] = v;
-    if ((e & 63) == 63) tree[index_slot_of_rank(e >> 6, P)] = v;
+// The arrays of one slot, and the one operation that fills them: entry e of the sorted buffer has value v.
+struct IndexSlot {
+  float* tree;
+  float* aux[kIndexMaxLevels];
+  float* buf;
+};
+__device__ __forceinline__ IndexSlot index_slot(uint32_t* index, const IndexLayout& L, int s) {
+  float* base = reinterpret_cast<float*>(index + kIndexHeaderWords + (size_t)s * L.slot_words);
+  IndexSlot t;
+  t.tree = base;
+#pragma unroll
+  for (int a = 0; a < kIndexMaxLevels; ++a) t.aux[a] = base + L.aux_off[a];
+  t.buf = base + L.buf_off;
+  return t;
+}
+__device__ __forceinline__ void index_put(const IndexSlot& t, const IndexShape& sh, int e, float v) {
+  t.buf[e] = v;
+  int m = 7;   // e ends an aligned group of 8^a entries iff its low 3a bits are all ones
+#pragma unroll
+  for (int a = 1; a <= kIndexMaxLevels; ++a) {
+    if (a > sh.A) break;
+    if ((e & m) != m) return;
+    t.aux[a - 1][e >> (3 * a)] = v;
+    m = (m << 3) | 7;
   }
-  for (int i = (n >> 3) + tid; i < 8 * ns; i += nthreads) aux[i] = qnan;             // groups of 8 that end beyond n
-  for (int r = (n >> 6) + tid; r < (1 << P) - 1; r += nthreads) tree[index_slot_of_rank(r, P)] = qnan;
+  if ((e & m) == m) t.tree[index_slot_of_rank(e >> (3 * (sh.A + 1)), sh.P)] = v;   // ends a group of 8^(A+1)
+}
+// NaN for the aux entries and tree nodes whose group ends beyond n (spread over `nthreads` callers).
+__device__ __forceinline__ void index_pad(const IndexSlot& t, const IndexShape& sh, int n, int tid, int nthreads) {
+  const float qnan = __uint_as_float(0x7FC00000u);
+#pragma unroll
+  for (int a = 1; a <= kIndexMaxLevels; ++a) {
+    if (a > sh.A) break;
+    const int first = n >> (3 * a), last = 8 * (n >> (3 * (a + 1))) + 8;
+    for (int i = first + tid; i < last; i += nthreads) t.aux[a - 1][i] = qnan;
+  }
+  for (int r = (n >> (3 * (sh.A + 1))) + tid; r < (1 << sh.P) - 1; r += nthreads) t.tree[index_slot_of_rank(r, sh.P)] = qnan;
+}
+// Header words of slot s.
+__device__ __forceinline__ void index_describe(uint32_t* index, int s, uint32_t n, const IndexShape& sh) {
+  uint32_t* d = index + 8 + 8 * s;
+  d[0] = n; d[1] = (uint32_t)sh.P; d[2] = (uint32_t)sh.A; d[3] = (uint32_t)sh.ns;
+}
+// The slot that describes fill n of an index laid out for `cap` entries, or -1.
+__device__ __forceinline__ int index_find(const uint32_t* __restrict__ index, uint32_t cap, uint32_t n) {
+  if (index[0] != kIndexMagic || index[1] != cap) return -1;
+  return index[8] == n ? 0 : (index[16] == n ? 1 : -1);
+}
+
+// Builds slot 0 of the index from src[0, n) (the caller's sorted buffer) and marks slot 1 empty.
+__global__ void __launch_bounds__(256)
+index_build_kernel(const float* __restrict__ src, int n, uint32_t cap, uint32_t* __restrict__ index) {
+  const IndexLayout L = index_layout(cap);
+  const IndexShape sh = index_shape(n);
+  const IndexSlot t = index_slot(index, L, 0);
+  const int tid = blockIdx.x * blockDim.x + threadIdx.x, nthreads = gridDim.x * blockDim.x;
+  if (tid == 0) {
+    index[0] = kIndexMagic;
+    index[1] = cap;
+    index_describe(index, 0, (uint32_t)n, sh);
+    index[16] = kIndexNoFill;
+  }
+  if (tid >= kIndexCountScratch && tid < kIndexCountScratch + 3 * kMaxAlphas + 1) index[tid] = 0u;
+  for (int e = tid; e < n; e += nthreads) index_put(t, sh, e, src[e]);
+  index_pad(t, sh, n, tid, nthreads);
 }
 
 template <int P>
-__device__ __forceinline__ void rank_four_indexed(const float (&s)[4], const float* __restrict__ sp,
-                                                  const float* __restrict__ aux, const float* __restrict__ calib, int n,
-                                                  uint32_t (&numer)[4]) {
+__device__ __forceinline__ void rank_four_indexed(const float (&s)[4], const float* __restrict__ sp, int A,
+                                                  const float* const (&aux)[kIndexMaxLevels],
+                                                  const float* __restrict__ calib, int n, uint32_t (&numer)[4]) {
   int g[4];
-  tree_descend<P>(s, sp, g);   // number of groups of 64 that lie entirely below the score
+  tree_descend<P>(s, sp, g);   // number of groups of 8^(A+1) that lie entirely below the score
   float w[4][8];
 #pragma unroll
-  for (int e = 0; e < 4; ++e)
-    asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                 : "=f"(w[e][0]), "=f"(w[e][1]), "=f"(w[e][2]), "=f"(w[e][3]), "=f"(w[e][4]), "=f"(w[e][5]), "=f"(w[e][6]), "=f"(w[e][7])
-                 : "l"(aux + 8 * g[e]));
-  int h[4];
+  for (int a = kIndexMaxLevels; a >= 1; --a) {
+    if (a > A) continue;
+    const float* __restrict__ lvl = aux[a - 1];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    int c = 0;
+    for (int e = 0; e < 4; ++e)
+      asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=f"(w[e][0]), "=f"(w[e][1]), "=f"(w[e][2]), "=f"(w[e][3]), "=f"(w[e][4]), "=f"(w[e][5]), "=f"(w[e][6]), "=f"(w[e][7])
+                   : "l"(lvl + 8 * g[e]));
 #pragma unroll
-    for (int i = 0; i < 7; ++i) c += (w[e][i] < s[e]) ? 1 : 0;   // the eighth is the group's splitter: not below
-    h[e] = 8 * g[e] + c;                                         // groups of 8 that lie entirely below the score
+    for (int e = 0; e < 4; ++e) {
+      int c = 0;
+#pragma unroll
+      for (int i = 0; i < 7; ++i) c += (w[e][i] < s[e]) ? 1 : 0;   // the eighth is the group's own splitter: not below
+      g[e] = 8 * g[e] + c;                                         // groups of 8^a that lie entirely below the score
+    }
   }
 #pragma unroll
   for (int e = 0; e < 4; ++e) {
-    // the last group may be cut short by n: its 32 bytes are still inside the 32-byte aligned span only if whole
-    if (8 * h[e] + 8 <= n) {
+    // the last group may be cut short by n: its 32 bytes are read in one piece only if it is whole
+    if (8 * g[e] + 8 <= n) {
       asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                    : "=f"(w[e][0]), "=f"(w[e][1]), "=f"(w[e][2]), "=f"(w[e][3]), "=f"(w[e][4]), "=f"(w[e][5]), "=f"(w[e][6]), "=f"(w[e][7])
-                   : "l"(calib + 8 * h[e]));
+                   : "l"(calib + 8 * g[e]));
     } else {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) w[e][i] = (8 * h[e] + i < n) ? __ldg(calib + 8 * h[e] + i) : __uint_as_float(0x7FC00000u);
+      for (int i = 0; i < 8; ++i) w[e][i] = (8 * g[e] + i < n) ? __ldg(calib + 8 * g[e] + i) : __uint_as_float(0x7FC00000u);
     }
   }
 #pragma unroll
@@ -513,33 +642,43 @@ __device__ __forceinline__ void rank_four_indexed(const float (&s)[4], const flo
     int c = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) c += (w[e][i] < s[e]) ? 1 : 0;
-    const int below = 8 * h[e] + c;
+    const int below = 8 * g[e] + c;
     numer[e] = (s[e] != s[e]) ? 0u : (uint32_t)(n - below) + 1u;   // NaN: no score
   }
 }
 
+// Every block takes one contiguous, equal share of the candidates (in groups of four), so that all SMs finish
+// together whatever the candidate count.
 template <int NA>
 __global__ void __launch_bounds__(kRankThreads)
-rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, const float* __restrict__ calib, int n, int P,
-                    const uint32_t* __restrict__ index, uint32_t* __restrict__ numer, float* __restrict__ pvalue,
-                    const FusedClassify fc, unsigned int* __restrict__ dev_status) {
+rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, int n, uint32_t* __restrict__ index,
+                    uint32_t* __restrict__ numer, float* __restrict__ pvalue, const FusedClassify fc,
+                    unsigned int* __restrict__ dev_status) {
   extern __shared__ float sp[];
-  // an index built for another fill of the buffer would give wrong ranks silently: refuse it
-  if (__ldg(index) != (uint32_t)n || __ldg(index + 1) != (uint32_t)P) {
+  pdl_launch_dependents();
+  pdl_wait();   // everything read below may come from the kernel before this one
+  // an index that does not describe this fill of the buffer would give wrong ranks silently: refuse it
+  const uint32_t cap = index[1];   // the capacity the index was laid out for, as its builder recorded it
+  const int slot = index_find(index, cap, (uint32_t)n);
+  if (slot < 0) {
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(dev_status, 8u);
     return;
   }
-  const float* const tree = reinterpret_cast<const float*>(index + kIndexHeaderWords);
-  const float* const aux = tree + kIndexTreeWords;
-  for (int t = threadIdx.x; t < (1 << P) - 1; t += kRankThreads) sp[t] = __ldg(tree + t);
+  const int P = (int)index[8 + 8 * slot + 1], A = (int)index[8 + 8 * slot + 2];
+  const IndexLayout L = index_layout(cap);
+  const float* const base = reinterpret_cast<const float*>(index + kIndexHeaderWords + (size_t)slot * L.slot_words);
+  const float* const aux[kIndexMaxLevels] = {base + L.aux_off[0], base + L.aux_off[1], base + L.aux_off[2]};
+  const float* const calib = base + L.buf_off;
+  for (int t = threadIdx.x; t < (1 << P) - 1; t += kRankThreads) sp[t] = __ldg(base + t);
   __syncthreads();
   StageTally<NA> tally;
   const float denom = (float)(n + 1);
   const float qnan = __uint_as_float(0x7FC00000u);
-  const int64_t per_block = (int64_t)kRankThreads * kRankPerThread;
-  for (int64_t base = (int64_t)blockIdx.x * per_block; base < Nc; base += (int64_t)gridDim.x * per_block) {
-    const int64_t j = base + (int64_t)threadIdx.x * kRankPerThread;
-    if (j >= Nc) continue;
+  const int64_t quads = (Nc + 3) >> 2;
+  const int64_t share = (quads + gridDim.x - 1) / gridDim.x;
+  const int64_t q_end = min(quads, ((int64_t)blockIdx.x + 1) * share);
+  for (int64_t q = (int64_t)blockIdx.x * share + threadIdx.x; q < q_end; q += kRankThreads) {
+    const int64_t j = 4 * q;
     float s[4];
     uint32_t r[4];
     const bool full = j + kRankPerThread <= Nc;
@@ -551,19 +690,19 @@ rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, const float* _
       for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
     }
     switch (P) {
-      case 1: rank_four_indexed<1>(s, sp, aux, calib, n, r); break;
-      case 2: rank_four_indexed<2>(s, sp, aux, calib, n, r); break;
-      case 3: rank_four_indexed<3>(s, sp, aux, calib, n, r); break;
-      case 4: rank_four_indexed<4>(s, sp, aux, calib, n, r); break;
-      case 5: rank_four_indexed<5>(s, sp, aux, calib, n, r); break;
-      case 6: rank_four_indexed<6>(s, sp, aux, calib, n, r); break;
-      case 7: rank_four_indexed<7>(s, sp, aux, calib, n, r); break;
-      case 8: rank_four_indexed<8>(s, sp, aux, calib, n, r); break;
-      case 9: rank_four_indexed<9>(s, sp, aux, calib, n, r); break;
-      case 10: rank_four_indexed<10>(s, sp, aux, calib, n, r); break;
-      case 11: rank_four_indexed<11>(s, sp, aux, calib, n, r); break;
-      case 12: rank_four_indexed<12>(s, sp, aux, calib, n, r); break;
-      default: rank_four_indexed<13>(s, sp, aux, calib, n, r); break;
+      case 1: rank_four_indexed<1>(s, sp, A, aux, calib, n, r); break;
+      case 2: rank_four_indexed<2>(s, sp, A, aux, calib, n, r); break;
+      case 3: rank_four_indexed<3>(s, sp, A, aux, calib, n, r); break;
+      case 4: rank_four_indexed<4>(s, sp, A, aux, calib, n, r); break;
+      case 5: rank_four_indexed<5>(s, sp, A, aux, calib, n, r); break;
+      case 6: rank_four_indexed<6>(s, sp, A, aux, calib, n, r); break;
+      case 7: rank_four_indexed<7>(s, sp, A, aux, calib, n, r); break;
+      case 8: rank_four_indexed<8>(s, sp, A, aux, calib, n, r); break;
+      case 9: rank_four_indexed<9>(s, sp, A, aux, calib, n, r); break;
+      case 10: rank_four_indexed<10>(s, sp, A, aux, calib, n, r); break;
+      case 11: rank_four_indexed<11>(s, sp, A, aux, calib, n, r); break;
+      case 12: rank_four_indexed<12>(s, sp, A, aux, calib, n, r); break;
+      default: rank_four_indexed<13>(s, sp, A, aux, calib, n, r); break;
     }
     float p[4] = {qnan, qnan, qnan, qnan};
     if (pvalue) {
@@ -572,7 +711,7 @@ rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, const float* _
     }
     emit_four<NA>(j, Nc, full, r, p, numer, pvalue, fc, tally);
   }
-  flush_tally<NA>(fc, tally);
+  flush_tally<NA>(fc, tally, index + kIndexCountScratch);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -626,113 +765,224 @@ classify_kernel(const uint32_t* __restrict__ numer, int64_t Nc, uint32_t k_alpha
   if (threadIdx.x < 3) {
     uint32_t t = 0;
     for (int i = 0; i < kClassifyThreads / 32; ++i) t += sh[threadIdx.x][i];
-    if (t) atomicAdd(counts + threadIdx.x, t);
+    if (gridDim.x == 1) counts[threadIdx.x] = t;   // a single block owns the counts: no zeroing beforehand
+    else if (t) atomicAdd(counts + threadIdx.x, t);
   }
 }
 
 // ---------------------------------------------------------------------------------------------
-// K5  sort of the new calibration scores by all-pairs ranking, spread over the whole GPU.  Every block
-// holds all k keys in shared memory (padded to a multiple of 128 with a key above every canonical key).
-// The slot of key j is the number of keys that sort before it: smaller keys, and equal keys that come earlier
-// in the input - one comparison per pair, key_i < key_j + (i < j).  A warp ranks four consecutive keys at a
-// time, so a 128-bit load of four other keys serves sixteen comparisons; those four others all come before or
-// all come after the warp's four, except in the one group that holds them.  k is at most kSortMaxK per launch.
+// K5 + K6  calibration update: sort of the new scores and merge-insert, in one kernel.
+//
+// The merged buffer is the stable merge of the old buffer (n entries, ascending) with the k new keys:
+//   old[e]  -> slot e + #{new <  old[e]}
+//   new x   -> slot #{old <= x} + #{new before x in sorted order}
+// No global sort of the new keys is needed for that.  The old buffer is cut into tiles of consecutive entries
+// [e0, e1); a new key x belongs to the tile that holds its insertion point, #{old <= x} in [e0, e1), which two
+// comparisons decide: old[e0 - 1] <= x < old[e1 - 1] (no lower test for the first tile, no upper test for the last).
+// A block that owns a tile reads all k new keys once, counts those below its range (c_below: they precede
+// everything the tile places), keeps its own (about k / tiles of them) in shared memory and sorts those few there;
+// keys of other tiles lie above its range and shift nothing here.  Then
+//   old[e], e in the tile  -> e + c_below + #{own keys <  old[e]}      (search among the few own keys)
+//   own key x, i-th of the sorted own keys -> e0 + #{tile entries <= x} + c_below + i   (search in the tile, in shared memory)
+// Equal keys are equal bit patterns after canonicalisation, so the order in which equal new keys are placed does
+// not show in the result.  One launch, no scratch besides the output, every global load and store coalesced.
+// A skewed batch (all new keys in one tile) only makes that block's sort longer, never wrong.
 // ---------------------------------------------------------------------------------------------
-constexpr int kSortMaxK = 16384;
-constexpr int kSortThreads = 256;
-constexpr int kSortKeysPerBlock = (kSortThreads / 32) * 4;
+constexpr int kSortMaxK = 16384;          // new keys per launch (larger batches are inserted slice by slice)
+constexpr int kMergeThreads = 1024;
+constexpr int kMergeTileMax = 8192;       // old entries per tile (32 KB of shared memory)
+constexpr int kMergeRankSortMax = 384;    // own keys up to this many are sorted by all-pairs ranking, more by a radix sort
 
-__global__ void __launch_bounds__(kSortThreads)
-sort_new_kernel(const float* __restrict__ new_scores, int k, uint32_t* __restrict__ sorted_keys) {
-  extern __shared__ __align__(16) uint32_t keys[];
-  const int kpad = (k + 127) & ~127;
-#pragma unroll 8
-  for (int t = threadIdx.x; t < kpad; t += kSortThreads)
-    keys[t] = t < k ? key_of_bits(canonical_bits(__ldg(new_scores + t))) : 0xFFFFFFFFu;
-  __syncthreads();
-  const int warps = kSortThreads / 32;
-  const int lane = threadIdx.x & 31;
-  for (int j0 = (blockIdx.x * warps + (threadIdx.x >> 5)) * 4; j0 < k; j0 += gridDim.x * warps * 4) {
-    const uint4 mine = *reinterpret_cast<const uint4*>(keys + j0);   // keys j0 .. j0 + 3 (padding beyond k)
-    const uint32_t kj[4] = {mine.x, mine.y, mine.z, mine.w};
-    int cnt[4] = {0, 0, 0, 0};
-    for (int i = lane * 4; i < kpad; i += 128) {
-      const uint4 q = *reinterpret_cast<const uint4*>(keys + i);
-      if (i != j0) {
-        const uint32_t earlier = i < j0 ? 1u : 0u;   // canonical keys stay below 0xFFC00001: no overflow
+constexpr int kRadixHistStride = 33;      // one column per warp, padded against bank conflicts
+
+// Block-wide radix sort (least significant byte first, four passes) of a[0, m), m <= 16384, by the kMergeThreads
+// threads of a block; b is a second array of the same size, both hold at least m rounded up to a multiple of
+// kMergeThreads words.  The sorted keys end in a.  hist: 256 * kRadixHistStride words, wsum: 32 words (shared).
+// Warp w owns the 32 E consecutive keys from w * 32 E on (E = keys per thread); in each pass a key's destination is
+// the number of keys with a smaller digit, plus those with the same digit in earlier warps, plus those with the
+// same digit earlier in its own warp, which keeps every pass stable.
+__device__ __forceinline__ void block_radix_sort(uint32_t* a, uint32_t* b, int m, uint32_t* hist, uint32_t* wsum) {
+  const int E = (m + kMergeThreads - 1) / kMergeThreads;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = m + threadIdx.x; i < E * kMergeThreads; i += kMergeThreads) a[i] = 0xFFFFFFFFu;   // sorts last
+  uint32_t* src = a;
+  uint32_t* dst = b;
+  const int entries = 256 * kRadixHistStride;
+  constexpr int kPer = (256 * kRadixHistStride + kMergeThreads - 1) / kMergeThreads;   // histogram words per thread in the scan
+  for (int shift = 0; shift < 32; shift += 8) {
+    for (int i = threadIdx.x; i < entries; i += kMergeThreads) hist[i] = 0u;
+    __syncthreads();
+    const uint32_t* mine = src + warp * 32 * E + lane;
+    uint32_t offs[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // two 16-bit offsets per word
 #pragma unroll
-        for (int y = 0; y < 4; ++y) {
-          const uint32_t t = kj[y] + earlier;
-          cnt[y] += (q.x < t) + (q.y < t) + (q.z < t) + (q.w < t);
+    for (int j = 0; j < 16; ++j) {
+      if (j < E) {
+        const uint32_t d = (mine[32 * j] >> shift) & 255u;
+        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
+        const uint32_t rank = (uint32_t)__popc(peers & ((1u << lane) - 1u));
+        uint32_t base = 0;
+        if (rank == 0) {   // first lane with this digit: column `warp` of the histogram is this warp's alone
+          base = hist[d * kRadixHistStride + warp];
+          hist[d * kRadixHistStride + warp] = base + (uint32_t)__popc(peers);
         }
-      } else {
-        const uint32_t qv[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-        for (int y = 0; y < 4; ++y)
-#pragma unroll
-          for (int x = 0; x < 4; ++x) cnt[y] += qv[x] < kj[y] + (x < y ? 1u : 0u);
+        base = __shfl_sync(0xFFFFFFFFu, base, __ffs((int)peers) - 1);
+        offs[j >> 1] |= (base + rank) << (16 * (j & 1));
+        __syncwarp();
       }
     }
+    __syncthreads();
+    // exclusive prefix sum of the histogram in digit-major, warp-minor order
+    {
+      const int first = threadIdx.x * kPer;
+      uint32_t sum = 0;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1)
+      for (int i = 0; i < kPer; ++i) sum += first + i < entries ? hist[first + i] : 0u;
+      uint32_t incl = sum;
 #pragma unroll
-      for (int y = 0; y < 4; ++y) cnt[y] += __shfl_xor_sync(0xFFFFFFFFu, cnt[y], o);
-    if (lane < 4 && j0 + lane < k) {
-      const int slot = lane == 0 ? cnt[0] : lane == 1 ? cnt[1] : lane == 2 ? cnt[2] : cnt[3];
-      sorted_keys[slot] = keys[j0 + lane];
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      if (lane == 31) wsum[warp] = incl;
+      __syncthreads();
+      uint32_t run = incl - sum;
+      for (int w = 0; w < warp; ++w) run += wsum[w];
+#pragma unroll
+      for (int i = 0; i < kPer; ++i) {
+        if (first + i < entries) {
+          const uint32_t v = hist[first + i];
+          hist[first + i] = run;
+          run += v;
+        }
+      }
     }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if (j < E) {
+        const uint32_t key = mine[32 * j];
+        const uint32_t d = (key >> shift) & 255u;
+        dst[hist[d * kRadixHistStride + warp] + ((offs[j >> 1] >> (16 * (j & 1))) & 0xFFFFu)] = key;
+      }
+    }
+    __syncthreads();
+    uint32_t* t = src; src = dst; dst = t;
   }
 }
 
-// ---------------------------------------------------------------------------------------------
-// K6  merge-insert.  Stable merge of the old buffer (n entries) with the sorted new keys (k):
-//   old[i]  -> slot i + #{new <  old[i]}
-//   new[j]  -> slot j + #{old <= new[j]}
-// written to `out` (n + k entries).  The new keys sit in shared memory for the first search; the
-// second searches the old buffer in global memory, 32 probes at a time.
-// ---------------------------------------------------------------------------------------------
-constexpr int kMergeThreads = 512;
+// Launch shape of the merge for n old entries on `sms` SMs: entries per tile and number of tiles (>= 1).
+__host__ __device__ inline void merge_tiling(int n, int sms, int& tile_len, int& tiles) {
+  const int rounds = (int)(((long long)n + (long long)sms * kMergeTileMax - 1) / ((long long)sms * kMergeTileMax));
+  const int want = sms * (rounds < 1 ? 1 : rounds);
+  tile_len = (n + want - 1) / want;
+  if (tile_len < 256) tile_len = 256;     // tiny buffers: a few tiles are enough
+  tiles = (n + tile_len - 1) / tile_len;
+  if (tiles < 1) tiles = 1;
+}
 
-__global__ void __launch_bounds__(kMergeThreads)
-merge_kernel(const float* __restrict__ old_buf, int n, const uint32_t* __restrict__ new_keys, int k,
-             float* __restrict__ out) {
-  extern __shared__ uint32_t nk[];
-#pragma unroll 8
-  for (int t = threadIdx.x; t < k; t += kMergeThreads) nk[t] = __ldg(new_keys + t);
-  __syncthreads();
-  // New keys first, one warp each: a 32-way search of the old buffer (every lane probes one of 32 evenly spaced
-  // entries, a ballot keeps the interval between the last "<=" and the first ">"), so the chain of dependent
-  // loads is log32(n) long instead of log2(n) and overlaps the bulk work below.
-  const int lane = threadIdx.x & 31;
-  const int warps_per_block = kMergeThreads / 32;
-  for (int j = blockIdx.x * warps_per_block + (threadIdx.x >> 5); j < k; j += gridDim.x * warps_per_block) {
-    const uint32_t key = nk[j];
-    int lo = 0, hi = n;  // the number of old keys <= key lies in [lo, hi]
-    while (hi > lo) {
-      const int width = hi - lo;
-      const int p = width >= 32 ? lo + (int)(((long long)width * (lane + 1)) >> 5) - 1 : lo + lane;
-      const bool le = p < hi && key_of_bits(canonical_bits(__ldg(old_buf + p))) <= key;
-      const int c = __popc(__ballot_sync(0xFFFFFFFFu, le));  // the predicate is true on a prefix of the lanes
-      const int p_prev = __shfl_sync(0xFFFFFFFFu, p, c > 0 ? c - 1 : 0);
-      const int p_next = __shfl_sync(0xFFFFFFFFu, p, c < 32 ? c : 31);
-      const int probes = width >= 32 ? 32 : width;
-      if (c > 0) lo = p_prev + 1;
-      if (c < probes) hi = p_next;
+// INDEXED == false: reads old_buf[0, n), writes the merged n + k entries to `out` (a scratch copy the host then
+// copies back: a tile's slots overlap the entries of the tiles after it).  INDEXED == true: the old entries are
+// read from the index slot that describes fill n, and every merged entry goes to the other slot (buffer copy, aux
+// entries, tree) and to `out`, which is the caller's buffer itself - nothing read here is written here, so there is
+// no copy back; `old_buf` is not used.
+// Dynamic shared memory: 4 * (2 * k2 + tile_len) bytes, k2 = k rounded up to a power of two, at least kMergeThreads.
+template <bool INDEXED>
+__global__ void __launch_bounds__(kMergeThreads, 1)
+merge_kernel(const float* __restrict__ old_buf, int n, const float* __restrict__ new_scores, int k, int k2, int tile_len,
+             int tiles, float* __restrict__ out, uint32_t* __restrict__ index, uint32_t cap,
+             unsigned int* __restrict__ dev_status) {
+  extern __shared__ uint32_t msm[];
+  uint32_t* const own = msm;             // [k2] this tile's new keys, as they come
+  uint32_t* const own_sorted = msm + k2; // [k2] the same, ascending
+  uint32_t* const tkeys = msm + 2 * k2;  // [tile_len] keys of the tile's old entries
+  __shared__ int own_count, below_count;
+  __shared__ uint32_t radix_hist[256 * kRadixHistStride], radix_wsum[kMergeThreads / 32];
+  pdl_launch_dependents();
+  pdl_wait();   // the new scores, the buffer and the index may come from the kernel before this one
+  IndexSlot dst{};
+  IndexShape sh{};
+  if (INDEXED) {
+    const int src = index_find(index, cap, (uint32_t)n);
+    if (src < 0) {   // no description of this fill: nothing is changed, the condition is reported
+      if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(dev_status, 8u);
+      return;
     }
-    if (lane == 0) out[j + lo] = __uint_as_float(bits_of_key(key));
+    const IndexLayout L = index_layout(cap);
+    old_buf = index_slot(index, L, src).buf;
+    dst = index_slot(index, L, src ^ 1);
+    sh = index_shape(n + k);
+    const int tid = blockIdx.x * kMergeThreads + threadIdx.x;
+    if (tid == 0) index_describe(index, src ^ 1, (uint32_t)(n + k), sh);
+    index_pad(dst, sh, n + k, tid, gridDim.x * kMergeThreads);
   }
-  // Old entries: each searches the sorted new keys in shared memory.
-  for (int e = blockIdx.x * kMergeThreads + threadIdx.x; e < n; e += gridDim.x * kMergeThreads) {
-    const uint32_t bits = canonical_bits(old_buf[e]);
-    const uint32_t key = key_of_bits(bits);
-    int lo = 0, len = k;  // number of new keys < key
-    while (len > 0) {
-      const int half = len >> 1;
-      const bool less = nk[lo + half] < key;
-      lo = less ? lo + half + 1 : lo;
-      len = less ? len - half - 1 : half;
+  auto emit = [&](int slot, uint32_t key) {
+    const float v = __uint_as_float(bits_of_key(key));
+    out[slot] = v;
+    if (INDEXED) index_put(dst, sh, slot, v);
+  };
+  for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
+    const int e0 = t * tile_len, e1 = min(n, e0 + tile_len), len = e1 - e0;
+    const bool first = e0 == 0, last = t == tiles - 1;
+    const uint32_t lo = first ? 0u : key_of_bits(canonical_bits(old_buf[e0 - 1]));
+    const uint32_t hi = last ? 0u : key_of_bits(canonical_bits(old_buf[e1 - 1]));
+    if (threadIdx.x == 0) { own_count = 0; below_count = 0; }
+    __syncthreads();
+    for (int i = threadIdx.x; i < len; i += kMergeThreads) tkeys[i] = key_of_bits(canonical_bits(old_buf[e0 + i]));
+    int below = 0;
+    for (int j = threadIdx.x; j < k; j += kMergeThreads) {
+      const uint32_t x = key_of_bits(canonical_bits(__ldg(new_scores + j)));
+      if (!first && x < lo) ++below;
+      else if (last || x < hi) own[atomicAdd(&own_count, 1)] = x;
     }
-    out[e + lo] = __uint_as_float(bits);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xFFFFFFFFu, below, o);
+    if ((threadIdx.x & 31) == 0 && below) atomicAdd(&below_count, below);
+    __syncthreads();
+    const int m = own_count, c_below = below_count;
+    // ---- sort the tile's own keys into own_sorted ----
+    if (m <= kMergeRankSortMax) {
+      // all-pairs: the slot of key i is the number of keys that sort before it (equal keys by position)
+      for (int i = threadIdx.x; i < m; i += kMergeThreads) {
+        const uint32_t x = own[i];
+        int r = 0;
+        for (int j = 0; j < m; ++j) {
+          const uint32_t y = own[j];
+          r += (y < x) || (y == x && j < i);
+        }
+        own_sorted[r] = x;
+      }
+      __syncthreads();
+    } else {
+      __syncthreads();   // every thread has read own_count
+      block_radix_sort(own, own_sorted, m, radix_hist, radix_wsum);
+      for (int i = threadIdx.x; i < m; i += kMergeThreads) own_sorted[i] = own[i];
+      __syncthreads();
+    }
+    // ---- place the own keys: e0 + #{tile entries <= x} + c_below + i ----
+    for (int i = threadIdx.x; i < m; i += kMergeThreads) {
+      const uint32_t x = own_sorted[i];
+      int p = 0, cnt = len;
+      while (cnt > 0) {
+        const int half = cnt >> 1;
+        const bool le = tkeys[p + half] <= x;
+        p = le ? p + half + 1 : p;
+        cnt = le ? cnt - half - 1 : half;
+      }
+      emit(e0 + p + c_below + i, x);
+    }
+    // ---- place the tile's old entries: e + c_below + #{own keys < old[e]} ----
+    for (int i = threadIdx.x; i < len; i += kMergeThreads) {
+      const uint32_t key = tkeys[i];
+      int p = 0, cnt = m;
+      while (cnt > 0) {
+        const int half = cnt >> 1;
+        const bool less = own_sorted[p + half] < key;
+        p = less ? p + half + 1 : p;
+        cnt = less ? cnt - half - 1 : half;
+      }
+      emit(e0 + i + c_below + p, key);
+    }
+    __syncthreads();   // shared memory is reused by the next tile
   }
 }
 
@@ -790,112 +1040,139 @@ classify_threshold_kernel(const float* __restrict__ scores, int64_t Nc, const fl
   if (threadIdx.x < 3) {
     uint32_t t = 0;
     for (int i = 0; i < kClassifyThreads / 32; ++i) t += sh[threadIdx.x][i];
-    if (t) atomicAdd(counts + threadIdx.x, t);
+    if (gridDim.x == 1) counts[threadIdx.x] = t;   // a single block owns the counts: no zeroing beforehand
+    else if (t) atomicAdd(counts + threadIdx.x, t);
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // Budget report: the positions of the samples in stage 3 (the target takes over), in input order, and their
-// number B.  Stream compaction in three launches: stage-3 count per tile of kIdsTile bytes; exclusive scan of the
-// tile counts by one block (which also writes B); every tile then recounts its bytes, 64 per thread, and writes
-// its positions from its offset on.  Everything is integer work in a fixed order: the result is unique.
+// number B.  A stream compaction in one pass over the stage bytes: a block takes tiles of kIdsTile bytes in the
+// order of a ticket counter, counts the stage-3 bytes of its tile, publishes that count, obtains the number of
+// stage-3 bytes in all earlier tiles by looking back over the published words of its predecessors (each word
+// holds a tile's own count or, once known, the count of everything up to and including it), and writes its
+// positions.  Tickets are drawn in launch order, so the block that owns an earlier tile is always running or
+// done: the look-back cannot wait on a block that has not started.  Every wait is bounded all the same.
+// Everything is integer work in a fixed order: the result is unique.
 // ---------------------------------------------------------------------------------------------
 constexpr int kIdsThreads = 256;
-constexpr int kIdsPerThread = 64;
-constexpr int kIdsTile = kIdsThreads * kIdsPerThread;   // 16384 stage bytes per block
+constexpr int kIdsPerThread = 32;                       // two 16-byte pieces per thread
+constexpr int kIdsTile = kIdsThreads * kIdsPerThread;   // 8192 stage bytes per tile
+constexpr unsigned long long kIdsOwnCount = 1ull << 32, kIdsPrefixKnown = 2ull << 32;
+constexpr int kIdsSpinLimit = 1 << 22;
 
-// Bit i of the result is set where byte i of the thread's 64 stage bytes is 3.
-__device__ __forceinline__ uint64_t stage3_mask(const uint8_t* __restrict__ stage, int64_t j, int64_t Nc, bool vec) {
-  uint64_t mask = 0;
-  if (vec && j + kIdsPerThread <= Nc) {
-    uint4 q[4];
+// Bit i of the result is set where byte i of the 16 stage bytes at stage + j is 3 (bytes beyond Nc are not).
+__device__ __forceinline__ uint32_t stage3_mask16(const uint8_t* __restrict__ stage, int64_t j, int64_t Nc, bool vec) {
+  uint32_t m16 = 0;
+  if (j >= Nc) return 0u;
+  if (vec && j + 16 <= Nc) {
+    const uint4 q = *reinterpret_cast<const uint4*>(stage + j);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-    for (int v = 0; v < 4; ++v) q[v] = *reinterpret_cast<const uint4*>(stage + j + 16 * v);
-#pragma unroll
-    for (int v = 0; v < 4; ++v) {
-      const uint32_t w[4] = {q[v].x, q[v].y, q[v].z, q[v].w};
-      uint32_t m16 = 0;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) m16 |= (((w[i >> 2] >> (8 * (i & 3))) & 0xFFu) == 3u ? 1u : 0u) << i;
-      mask |= (uint64_t)m16 << (16 * v);
-    }
+    for (int i = 0; i < 16; ++i) m16 |= (((w[i >> 2] >> (8 * (i & 3))) & 0xFFu) == 3u ? 1u : 0u) << i;
   } else {
-    for (int i = 0; i < kIdsPerThread && j + i < Nc; ++i) mask |= (uint64_t)(stage[j + i] == 3 ? 1u : 0u) << i;
+    for (int i = 0; i < 16 && j + i < Nc; ++i) m16 |= (stage[j + i] == 3 ? 1u : 0u) << i;
   }
-  return mask;
+  return m16;
 }
 
-// Exclusive prefix sum of one value per thread over a block of kIdsThreads; *total gets the block's sum.
-__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* total) {
-  __shared__ uint32_t warp_sum[kIdsThreads / 32];
-  __shared__ uint32_t block_sum;
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// state: one word per tile (zero before the launch), ticket: one counter (zero before the launch); both unused
+// (may be nullptr) when there is a single tile.
+__global__ void __launch_bounds__(kIdsThreads)
+takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int tiles, bool vec,
+                    unsigned long long* __restrict__ state, unsigned int* __restrict__ ticket,
+                    int32_t* __restrict__ ids, int64_t ids_cap, uint32_t* __restrict__ count,
+                    unsigned int* __restrict__ dev_status) {
+  __shared__ int32_t staged[kIdsTile];
+  __shared__ uint32_t warp_total[kIdsThreads / 32];
+  __shared__ uint32_t tile_sh, prefix_sh;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t incl = v;
+  for (;;) {
+    if (threadIdx.x == 0) tile_sh = tiles == 1 ? blockIdx.x : atomicAdd(ticket, 1u);
+    __syncthreads();
+    const int tile = (int)tile_sh;
+    if (tile >= tiles) return;
+    // A warp covers 1024 consecutive bytes as two rows of 512: lane l holds bytes [16 l, 16 l + 16) of each row, so
+    // every load instruction of the warp reads 512 contiguous bytes.
+    const int64_t warp_base = (int64_t)tile * kIdsTile + (int64_t)warp * (kIdsPerThread * 32);
+    uint32_t m[2], excl[2], row_total[2];
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-    if (lane >= o) incl += up;
-  }
-  if (lane == 31) warp_sum[warp] = incl;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t run = 0;
-    for (int w = 0; w < kIdsThreads / 32; ++w) {
-      const uint32_t t = warp_sum[w];
-      warp_sum[w] = run;
-      run += t;
+    for (int r = 0; r < 2; ++r) {
+      m[r] = stage3_mask16(stage, warp_base + r * 512 + lane * 16, Nc, vec);
+      uint32_t incl = (uint32_t)__popc(m[r]);
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      excl[r] = incl - (uint32_t)__popc(m[r]);
+      row_total[r] = __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
-    block_sum = run;
-  }
-  __syncthreads();
-  const uint32_t excl = warp_sum[warp] + incl - v;
-  *total = block_sum;
-  __syncthreads();   // the shared words may be reused by the next call
-  return excl;
-}
-
-__global__ void __launch_bounds__(kIdsThreads)
-takeover_count_kernel(const uint8_t* __restrict__ stage, int64_t Nc, bool vec, uint32_t* __restrict__ tile_count) {
-  const int64_t j = (int64_t)blockIdx.x * kIdsTile + (int64_t)threadIdx.x * kIdsPerThread;
-  uint32_t c = j < Nc ? (uint32_t)__popcll(stage3_mask(stage, j, Nc, vec)) : 0u;
+    if (lane == 0) warp_total[warp] = row_total[0] + row_total[1];
+    __syncthreads();
+    uint32_t warp_off = 0, total = 0;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-  __shared__ uint32_t sh[kIdsThreads / 32];
-  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = c;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t t = 0;
-    for (int w = 0; w < kIdsThreads / 32; ++w) t += sh[w];
-    tile_count[blockIdx.x] = t;
-  }
-}
-
-// One block: tile_count[t] <- sum of the counts of the tiles before t; *count <- the sum of all (may be nullptr).
-__global__ void __launch_bounds__(kIdsThreads)
-takeover_scan_kernel(uint32_t* __restrict__ tile_count, int tiles, uint32_t* __restrict__ count) {
-  uint32_t carry = 0;
-  for (int base = 0; base < tiles; base += kIdsThreads) {
-    const int t = base + threadIdx.x;
-    const uint32_t v = t < tiles ? tile_count[t] : 0u;
-    uint32_t total;
-    const uint32_t excl = block_exclusive_scan(v, &total);
-    if (t < tiles) tile_count[t] = carry + excl;
-    carry += total;
-  }
-  if (threadIdx.x == 0 && count != nullptr) *count = carry;
-}
-
-__global__ void __launch_bounds__(kIdsThreads)
-takeover_write_kernel(const uint8_t* __restrict__ stage, int64_t Nc, bool vec, const uint32_t* __restrict__ tile_offset,
-                      int32_t* __restrict__ ids, int64_t ids_cap) {
-  const int64_t j = (int64_t)blockIdx.x * kIdsTile + (int64_t)threadIdx.x * kIdsPerThread;
-  const uint64_t mask = j < Nc ? stage3_mask(stage, j, Nc, vec) : 0ull;
-  uint32_t total;
-  const uint32_t excl = block_exclusive_scan((uint32_t)__popcll(mask), &total);
-  int64_t pos = (int64_t)tile_offset[blockIdx.x] + excl;
-  for (uint64_t m = mask; m != 0ull; m &= m - 1ull) {
-    if (pos < ids_cap) ids[pos] = (int32_t)(j + (__ffsll((long long)m) - 1));
-    ++pos;
+    for (int w = 0; w < kIdsThreads / 32; ++w) {
+      const uint32_t t = warp_total[w];
+      warp_off += w < warp ? t : 0u;
+      total += t;
+    }
+    // positions of this tile, in order, into shared memory
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      uint32_t loc = warp_off + (r ? row_total[0] : 0u) + excl[r];
+      const int32_t first = (int32_t)(warp_base + r * 512 + lane * 16);
+      for (uint32_t mm = m[r]; mm != 0u; mm &= mm - 1u) staged[loc++] = first + (__ffs((int)mm) - 1);
+    }
+    // number of stage-3 bytes in all earlier tiles
+    if (warp == 0) {
+      uint32_t prefix = 0;
+      if (tiles > 1) {
+        if (lane == 0) {
+          __threadfence();
+          atomicExch(state + tile, (tile == 0 ? kIdsPrefixKnown : kIdsOwnCount) | total);
+        }
+        int spins = 0;
+        for (int p0 = tile - 1; p0 >= 0; ) {
+          const int p = p0 - lane;
+          const unsigned long long w = p >= 0 ? ld_relaxed_u64(state + p) : kIdsPrefixKnown;
+          const uint32_t ready = __ballot_sync(0xFFFFFFFFu, (w >> 32) != 0ull);
+          if (ready != 0xFFFFFFFFu) {
+            if (++spins > kIdsSpinLimit) {   // cannot happen with tickets in launch order; give up rather than hang
+              if (lane == 0) atomicOr(dev_status, 2u);
+              break;
+            }
+            __nanosleep(20);
+            continue;
+          }
+          const uint32_t known = __ballot_sync(0xFFFFFFFFu, (w >> 32) == 2ull);
+          const int stop = known ? __ffs((int)known) - 1 : 31;   // nearest predecessor whose prefix is known
+          uint32_t v = lane <= stop ? (uint32_t)w : 0u;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+          prefix += v;
+          if (known) break;
+          p0 -= 32;
+        }
+        if (lane == 0 && tile > 0) atomicExch(state + tile, kIdsPrefixKnown | (unsigned long long)(prefix + total));
+      }
+      if (lane == 0) {
+        prefix_sh = prefix;
+        if (tile == tiles - 1 && count != nullptr) *count = prefix + total;
+      }
+    }
+    __syncthreads();
+    const int64_t prefix = prefix_sh;
+    for (uint32_t t = threadIdx.x; t < total; t += kIdsThreads)
+      if (prefix + t < ids_cap) ids[prefix + t] = staged[t];
+    if (tiles == 1) return;
+    __syncthreads();   // the shared words are reused by the next tile
   }
 }
 
@@ -1030,7 +1307,7 @@ classify_conditional_kernel(const uint32_t* __restrict__ numer, const uint32_t* 
   for (int i = 0; i < 3; ++i) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) c[i] += __shfl_xor_sync(0xFFFFFFFFu, c[i], o);
-    if ((threadIdx.x & 31) == 0 && c[i]) atomicAdd(counts + i, c[i]);
+    if ((threadIdx.x & 31) == 0 && c[i]) atomicAdd(counts + i, c[i]);   // counts are zeroed by the host
   }
 }
 

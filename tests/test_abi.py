@@ -61,17 +61,18 @@ def test_argument_errors_need_no_device():
     assert lib.atts_score_logprob(None, None, None, None, 8, 64, 100, 1, 0, None, None, None, 0, None) == 1
     assert lib.atts_last_device_status(None, None) == 1
     assert lib.atts_calib_index_bytes(524223, ctypes.byref(sz)) == 0 and sz.value % 256 == 0 and sz.value >= 4 * (8192 + 8 * 8191)
-    assert lib.atts_calib_index_bytes(524224, ctypes.byref(sz)) == 2                        # too large for an index
+    assert lib.atts_calib_index_bytes((1 << 24) - 2, ctypes.byref(sz)) == 0 and sz.value >= 8 * ((1 << 24) - 2)
+    assert lib.atts_calib_index_bytes((1 << 24) - 1, ctypes.byref(sz)) == 2                 # beyond the buffer API's range
     assert lib.atts_calib_index_bytes(10, None) == 1
     assert lib.atts_takeover_ids_workspace_bytes(1 << 20, ctypes.byref(sz)) == 0 and sz.value >= 4 * 64 and sz.value % 256 == 0
     assert lib.atts_takeover_ids_workspace_bytes(-1, ctypes.byref(sz)) == 2
     assert lib.atts_takeover_ids(None, 8, None, 8, None, None, 0, None) == 1
     assert lib.atts_takeover_ids(None, 8, None, -1, None, None, 0, None) == 2
     assert lib.atts_calib_index_build(None, 10, None, 0, None) == 1
-    assert lib.atts_calib_index_build(None, 1 << 20, None, 0, None) == 2
+    assert lib.atts_calib_index_build(None, 1 << 24, None, 0, None) == 2
     assert lib.atts_calib_update_indexed(None, 10, 20, None, 5, None, None, 0, None, 0, None) == 1
     assert lib.atts_rank_classify_indexed(None, 4, None, 0, None, None, 5, None, None, None, None, None) == 6
-    assert lib.atts_rank_classify_indexed(None, 4, None, 1 << 20, None, None, 0, None, None, None, None, None) == 2
+    assert lib.atts_rank_classify_indexed(None, 4, None, 1 << 24, None, None, 0, None, None, None, None, None) == 2
 
 
 def test_no_device_means_error_not_fallback():

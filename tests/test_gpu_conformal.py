@@ -337,7 +337,8 @@ def _index_for(calib_dev, n, cap=None):
 
 
 @pytest.mark.parametrize("Nc,n", [(1 << 17, 8192), (100003, 8255), (1 << 16, 65536), (70001, 65543), (1 << 18, 327680),
-                                   (16384, 524223), (20000, 100), (100, 70000), (0, 9000)])
+                                   (16384, 524223), (20000, 100), (100, 70000), (0, 9000), (16384, 65527), (16384, 65528),
+                                   (1 << 16, 524224), (1 << 15, 4193791), (1 << 15, 4193792)])
 def test_indexed_rank_equals_definition_and_plain_call(Nc, n):
     """The indexed rank gives the numerators and p-value bits of the definition, on smooth data, on heavily tied data
     and with special values at both ends of the buffer, with and without fused thresholds."""
@@ -406,7 +407,7 @@ def test_stale_index_is_refused_and_argument_errors():
     n, Nc = 20000, 1 << 15
     calib = np.sort(inputs.lognormal_scores(90, n + 64))
     c, s = dev(calib), dev(inputs.lognormal_scores(91, Nc))
-    ix = _index_for(c, n, n + 64)
+    ix = _index_for(c, n, n + 64 + 5000)
     numer = poison((Nc,), torch.int32)
     binding.rank_classify_indexed(s, c, n + 64, ix, (), numer)           # index describes n, not n + 64
     with pytest.raises(binding.AttsError) as err:
@@ -414,9 +415,97 @@ def test_stale_index_is_refused_and_argument_errors():
     assert err.value.status == 11
     assert np.all(host_u32(numer) == 0xFFFFFFFF)                         # nothing was written
     assert binding.last_device_status() == 0                             # the bit was cleared
-    with pytest.raises(binding.AttsError) as err:                        # buffer not 32-byte aligned
-        binding.rank_classify_indexed(s, c[1:], n, ix, (), numer)
-    assert err.value.status == 3
+    # an update through an index that does not describe the fill it starts from changes nothing and is reported
+    buf = poison((n + 64 + 5000,), torch.float32)
+    buf[:n + 64] = c
+    new = dev(inputs.lognormal_scores(92, 5000))
+    binding.calib_update_indexed(buf, n + 64, new, ix, workspace(binding.calib_workspace_bytes(n + 64, 5000)))
+    with pytest.raises(binding.AttsError) as err:
+        binding.last_device_status()
+    assert err.value.status == 11
+    assert np.array_equal(f32_bits(buf[:n + 64]), f32_bits(calib)) and np.all(f32_bits(buf[n + 64:]) == 0xFFFFFFFF)
+    # the fill it does describe is still served, from the index's own copy of the buffer
+    binding.rank_classify_indexed(s, c, n, ix, (), numer)
+    torch.cuda.synchronize()
+    assert np.array_equal(host_u32(numer), orc.conformal_numer_sorted(inputs.lognormal_scores(91, Nc), calib[:n]))
     with pytest.raises(binding.AttsError) as err:                        # index too small for this n
         binding.calib_index_build(c, n + 64, ix[:1024])
     assert err.value.status == 4
+
+
+def test_indexed_update_may_overlap_the_rank_of_the_fill_it_starts_from():
+    """Rank of fill n on one stream, the update n -> n + k on another, with no ordering between them: the rank sees the
+    buffer as it was (ranks against the old fill), the update leaves the new one; the next rank waits for the update,
+    the next update for this rank.  Several steps, every result against the oracle."""
+    Nc, n, k, steps = 1 << 17, 90000, 4096, 5
+    calib = np.sort(inputs.lognormal_scores(310, n))
+    scores = inputs.lognormal_scores(311, Nc)
+    news = [inputs.lognormal_scores(312 + t, k) for t in range(steps)]
+    s, nws = dev(scores), [dev(x) for x in news]
+    cap = n + k * steps
+    buf = poison((cap,), torch.float32)
+    buf[:n] = dev(calib)
+    ix = _index_for(buf, n, cap)
+    ws = workspace(binding.calib_workspace_bytes(cap, k))
+    numers = [poison((Nc,), torch.int32) for _ in range(steps)]
+    main, side = torch.cuda.current_stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    ranked, merged = [], []
+    fill = n
+    for t in range(steps):
+        if t:
+            main.wait_event(merged[t - 1])                   # the rank of fill n_t needs the update that produced it
+        binding.rank_classify_indexed(s, buf, fill, ix, (), numers[t])
+        ev = torch.cuda.Event()
+        ev.record(main)
+        ranked.append(ev)
+        with torch.cuda.stream(side):
+            if t:
+                side.wait_event(ranked[t - 1])               # this update overwrites what the previous rank read
+            fill = binding.calib_update_indexed(buf, fill, nws[t], ix, ws)
+            ev = torch.cuda.Event()
+            ev.record(side)
+            merged.append(ev)
+    torch.cuda.synchronize()
+    want = calib
+    for t in range(steps):
+        assert np.array_equal(host_u32(numers[t]), orc.conformal_numer_sorted(scores, want)), t
+        want = orc.calib_update(want, news[t])
+    assert fill == cap and np.array_equal(f32_bits(buf), f32_bits(want))
+    assert binding.last_device_status() == 0
+
+
+@pytest.mark.parametrize("n,k", [(70000, 4096), (40000, 16384), (300000, 20000), (5000, 600), (0, 3000), (100000, 385)])
+def test_update_with_skewed_batches(n, k):
+    """New scores that all fall into one stretch of the buffer (beyond its largest entry, below its smallest, one
+    repeated value, a narrow band, everything NaN): the block that owns that stretch sorts them all.  Plain and
+    indexed update against the oracle."""
+    calib = np.sort(inputs.lognormal_scores(400 + n, n))
+    top = float(calib[-1]) if n else 1.0
+    mid = float(calib[n // 2]) if n else 1.0
+    batches = {
+        "above": top + 1.0 + inputs.lognormal_scores(401, k),
+        "below": -inputs.lognormal_scores(402, k),
+        "equal": np.full(k, mid, np.float32),
+        "band": (mid + 1e-4 * inputs.lognormal_scores(403, k)).astype(np.float32),
+        "nan": np.full(k, np.nan, np.float32),
+        "two_values": np.where(np.arange(k) % 2 == 0, np.float32(mid), np.float32(top + 2.0)).astype(np.float32),
+    }
+    for name, new in batches.items():
+        new = new.astype(np.float32)
+        want = orc.calib_update(calib, new)
+        for indexed in (False, True):
+            buf = poison((n + k + 5,), torch.float32)
+            if n:
+                buf[:n] = dev(calib)
+            ws = workspace(binding.calib_workspace_bytes(n, k))
+            if indexed:
+                ix = _index_for(buf, n, n + k)
+                n2 = binding.calib_update_indexed(buf, n, dev(new), ix, ws)
+            else:
+                n2 = binding.calib_update(buf, n, dev(new), ws)
+            torch.cuda.synchronize()
+            assert n2 == n + k
+            assert np.array_equal(f32_bits(buf[:n2]), f32_bits(want)), (name, indexed)
+            assert np.all(f32_bits(buf[n2:]) == 0xFFFFFFFF), (name, indexed)
+    assert binding.last_device_status() == 0

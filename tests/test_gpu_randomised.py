@@ -35,7 +35,7 @@ def draw(rng, n, kind):
 def test_randomised_rank_index_update_and_budget_report():
     rng = np.random.default_rng(777)
     for case in range(48):
-        n = int(rng.choice([1, 2, 3, 100, 4095, 4096, 8191, 8192, 8193, 20000, 65536, 100001, 300000, 524223]))
+        n = int(rng.choice([1, 2, 3, 100, 4095, 4096, 8191, 8192, 8193, 20000, 65527, 65536, 100001, 300000, 524223, 524224, 1000003]))
         Nc = int(rng.choice([1, 17, 4096, 16384, 65536, 65536 + 48, 200000]))
         kc, ks = int(rng.integers(0, 5)), int(rng.integers(0, 5))
         calib = orc.calib_update(np.zeros(0, np.float32), draw(rng, n, kc))
@@ -65,11 +65,12 @@ def test_randomised_rank_index_update_and_budget_report():
         want_ids = np.flatnonzero(orc.classify(want, n, alphas[0])[0] == 3)
         assert host_u32(count)[0] == want_ids.size and np.array_equal(ids.cpu().numpy()[:want_ids.size], want_ids)
         k = int(rng.choice([0, 1, 64, 4096, 5000, 20000]))
-        if n + k <= 524223:
+        if True:
             new = draw(rng, k, int(rng.integers(0, 5)))
             buf = poison((n + k + 8,), torch.float32)
             buf[:n] = c
             index2 = workspace(binding.calib_index_bytes(n + k))
+            binding.calib_index_build(buf, n, index2)
             n2 = binding.calib_update_indexed(buf, n, dev(new) if k else None, index2,
                                               workspace(binding.calib_workspace_bytes(n, k)))
             want_buf = orc.calib_update(calib, new)
