@@ -109,34 +109,49 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def oracle_step(orc, Hb, Wb, ids, rows, N, calib, alpha):
-    """One pass of the oracle over a bounded sample: `rows` token rows scored, then the conformal steps."""
-    lp = orc.token_logprob(Hb[:rows], Wb, ids[:rows])
-    per = max(rows // N, 1)
-    off = np.minimum(np.arange(N + 1) * per, rows).astype(np.int32)
-    sc = orc.sample_score(lp, off).astype(np.float32)
+def oracle_rows_plan(M: int, T: int, whole_samples: int, scattered: int, seed: int) -> np.ndarray:
+    """Token rows the oracle scores out of a batch of M: the first `whole_samples` samples completely, plus
+    `scattered` rows drawn by a seeded permutation from the rest (every row spans the whole vocabulary and hidden
+    dimension, so every tile column is exercised by every row)."""
+    head = np.arange(min(whole_samples * T, M))
+    rest = np.arange(head.size, M)
+    pick = np.random.default_rng(seed).permutation(rest)[:scattered] if rest.size else rest
+    return np.concatenate([head, np.sort(pick)]).astype(np.int64)
+
+
+def oracle_step(orc, H_rows, Wb, ids_rows, whole_rows, T, scores_rest, calib, alpha):
+    """One pass of the oracle over a bounded sample: the given token rows scored (the first `whole_rows` of them are
+    whole samples of T tokens and give sample scores), then rank / p-value / stage / insert on the batch's scores
+    (`scores_rest` stands in for the samples the oracle did not score)."""
+    lp = orc.token_logprob(H_rows, Wb, ids_rows)
+    own = np.zeros(0, np.float32)
+    if whole_rows:
+        off = (np.arange(whole_rows // T + 1) * T).astype(np.int32)
+        own = orc.sample_score(lp[:whole_rows], off).astype(np.float32)
+    sc = np.concatenate([own, np.asarray(scores_rest, np.float32)])
     numer = orc.conformal_numer_sorted(sc, calib)
     orc.pvalue(numer, calib.size)
     orc.classify(numer, calib.size, alpha)
     return orc.calib_update(calib, sc[~np.isnan(sc)])
 
 
-def oracle_conformal_steps(orc, steps_timed=16):
-    """The oracle on the first steps of the conformal-only workload: rank, p-values, three thresholds, insert."""
+def oracle_conformal_steps(orc):
+    """The oracle on the whole conformal-only workload: rank, p-values, three thresholds and insert, 64 steps."""
     cfg = inputs.CONFORMAL_STRESS
+    steps = cfg["steps"]
     scores = inputs.lognormal_scores(inputs.BASE_SEED + 1, cfg["Nc"])
     calib = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, cfg["n0"]))
-    news = [inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, cfg["k"]) for t in range(steps_timed)]
+    news = [inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, cfg["k"]) for t in range(steps)]
     t0 = time.perf_counter()
-    for t in range(steps_timed):
+    for t in range(steps):
         numer = orc.conformal_numer_sorted(scores, calib)
         orc.pvalue(numer, calib.size)
         for alpha in cfg["alphas"]:
             orc.classify(numer, calib.size, alpha)
         calib = orc.calib_update(calib, news[t])
     dt = time.perf_counter() - t0
-    return {"value": cfg["Nc"] * steps_timed / dt, "unit": "p-values/s", "cores": 1, "kind": "oracle",
-            "sample": f"first {steps_timed} of {cfg['steps']} steps of the conformal-only workload in {dt:.1f} s"}
+    return {"value": cfg["Nc"] * steps / dt, "unit": "p-values/s", "cores": 1, "kind": "oracle",
+            "sample": f"all {steps} steps of the conformal-only workload in {dt:.1f} s"}
 
 
 def blas_threads():
@@ -156,143 +171,48 @@ def run_reference(args):
     from oracle import atts_oracle as orc
     c = inputs.CONFIGS[args.workload]
     N, T, d, V, n0 = c["N"], c["T"], c["d"], c["V"], c["n"]
+    M = N * T
     rows = args.oracle_rows
     Wb = inputs.lm_head(inputs.BASE_SEED, V, d)
-    Hb = inputs.hidden(inputs.BASE_SEED + 1, N * T, d, 0, rows)
-    ids = inputs.zipf_ids(inputs.BASE_SEED + 2, N * T, V)
-    # the oracle cannot afford to score 4096 calibration samples: a LogNormal-shaped stand-in near the NLL scale
+    # token rows scattered over the batch: a few rows from each of a few seeded slabs (a slab is what the input
+    # generator can reproduce on its own)
+    rng = np.random.default_rng(inputs.BASE_SEED + 9)
+    n_slabs = -(-M // inputs.SLAB_ROWS)
+    slabs = np.sort(rng.choice(n_slabs, size=min(n_slabs, max(1, rows // 16)), replace=False))
+    per = -(-rows // slabs.size)
+    picks, parts = [], []
+    for j in slabs:
+        a0, b0 = j * inputs.SLAB_ROWS, min((j + 1) * inputs.SLAB_ROWS, M)
+        loc = np.sort(rng.choice(b0 - a0, size=min(per, b0 - a0), replace=False))
+        parts.append(inputs.hidden(inputs.BASE_SEED + 1, M, d, a0, b0)[loc])
+        picks.append(a0 + loc)
+    idx = np.concatenate(picks)[:rows]
+    Hb = np.concatenate(parts)[:rows]
+    ids = inputs.zipf_ids(inputs.BASE_SEED + 2, M, V)[idx]
+    rows = idx.size
+    # the oracle cannot afford to score 4096 calibration samples or the other samples of the batch: LogNormal-shaped
+    # stand-ins near the NLL scale feed the conformal steps
     calib = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 5, n0)) + np.float32(11.0)
+    rest = inputs.lognormal_scores(inputs.BASE_SEED + 6, N) + np.float32(11.0)
     for _ in range(args.warmup):
-        calib = oracle_step(orc, Hb, Wb, ids, rows, N, calib, ALPHA)
+        calib = oracle_step(orc, Hb, Wb, ids, 0, T, rest, calib, ALPHA)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        calib = oracle_step(orc, Hb, Wb, ids, rows, N, calib, ALPHA)
+        calib = oracle_step(orc, Hb, Wb, ids, 0, T, rest, calib, ALPHA)
     dt = time.perf_counter() - t0
     value = rows * args.steps / dt
-    sample = f"{rows} of {N * T} token rows per step (full d and V), then rank/classify/update on N={N} scores"
+    sample = (f"{rows} of {M} token rows per step, scattered over the batch by a seeded choice (full d and V), then "
+              f"rank/classify/update on N={N} scores")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"32B-target shape N={N} T={T} d={d} V={V} n={n0} alpha={ALPHA}", "sample": sample},
+        "config": {"workload": f"{args.workload.upper()}-target shape N={N} T={T} d={d} V={V} n={n0} alpha={ALPHA}", "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
-
-
-def conformal_stress(torch, binding, peaks):
-    """Extra figures on the conformal-only workload: 2^20 candidates against a buffer growing from 65,536 by 4,096 a
-    step, three alphas; kernel times by CUDA events (the working set is L2-resident)."""
-    cfg = inputs.CONFORMAL_STRESS
-    Nc, n0, k, steps = cfg["Nc"], cfg["n0"], cfg["k"], cfg["steps"]
-    dev = "cuda"
-    scores = torch.from_numpy(inputs.lognormal_scores(inputs.BASE_SEED + 1, Nc)).to(dev)
-    calib0 = torch.from_numpy(np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, n0))).to(dev)
-    news = [torch.from_numpy(inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, k)).to(dev) for t in range(steps)]
-    cap = n0 + k * steps
-    buf = torch.empty(cap, device=dev)
-    numer = torch.empty(Nc, dtype=torch.int32, device=dev)
-    p = torch.empty(Nc, device=dev)
-    stage = torch.empty(Nc, dtype=torch.uint8, device=dev)
-    counts = torch.empty(3, dtype=torch.int32, device=dev)
-    stage3 = torch.empty((len(cfg["alphas"]), Nc), dtype=torch.uint8, device=dev)
-    counts3 = torch.empty((len(cfg["alphas"]), 3), dtype=torch.int32, device=dev)
-    ws = torch.empty(binding.calib_workspace_bytes(cap, k), dtype=torch.uint8, device=dev)
-
-    index = torch.empty(binding.calib_index_bytes(cap), dtype=torch.uint8, device=dev)
-
-    def sequence_plain():
-        buf[:n0] = calib0
-        n = n0
-        for t in range(steps):
-            binding.rank_classify(scores, buf, n, cfg["alphas"], numer, p, stage3, counts3)
-            n = binding.calib_update(buf, n, news[t], ws)
-        return n
-
-    def sequence():
-        # the calibration state is the buffer and its search index; every update rebuilds the index
-        buf[:n0] = calib0
-        binding.calib_index_build(buf, n0, index)
-        n = n0
-        for t in range(steps):
-            binding.rank_classify_indexed(scores, buf, n, index, cfg["alphas"], numer, p, stage3, counts3)
-            n = binding.calib_update_indexed(buf, n, news[t], index, ws)
-        return n
-
-    graph_ms = make_graph_timer(torch)
-    ms_seq_plain = graph_ms(sequence_plain)
-    ms_seq = graph_ms(sequence)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    eager = []
-    for _ in range(3):
-        e0.record()
-        sequence()
-        e1.record()
-        torch.cuda.synchronize()
-        eager.append(e0.elapsed_time(e1))
-
-    n_end = cap - k
-    ms_rank = graph_ms(lambda: binding.conformal_rank(scores, buf, n_end, numer, p), reps=20)
-    ms_cls = graph_ms(lambda: binding.classify(numer, n_end, 0.1, stage, counts), reps=20)
-    ms_upd = graph_ms(lambda: binding.calib_update(buf, n_end, news[0], ws), reps=20)
-    ms_fused = graph_ms(lambda: binding.rank_classify(scores, buf, n_end, cfg["alphas"], numer, p, stage3, counts3), reps=20)
-    binding.calib_index_build(buf, n_end, index)
-    ms_fused_ix = graph_ms(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, cfg["alphas"], numer, p, stage3,
-                                                                 counts3), reps=20)
-    ms_upd_ix = graph_ms(lambda: binding.calib_update_indexed(buf, n_end, news[0], index, ws), reps=20)
-    # The same calls with a cold L2: 512 MB are written between repetitions, one call is timed by events (the events'
-    # own few microseconds are inside), median of 9.
-    scrub = torch.empty(128 << 20, dtype=torch.float32, device=dev)
-
-    def cold_us(fn):
-        ts = []
-        for _ in range(9):
-            scrub.fill_(1.0)
-            torch.cuda.synchronize()
-            e0.record()
-            fn()
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1) * 1e3)
-        return float(np.median(ts))
-
-    binding.calib_index_build(buf, n_end, index)   # the timed update above left the index of a larger fill
-    cold = {
-        "rank_classify_indexed_us": cold_us(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, cfg["alphas"],
-                                                                              numer, p, stage3, counts3)),
-        "rank_classify_us": cold_us(lambda: binding.rank_classify(scores, buf, n_end, cfg["alphas"], numer, p, stage3, counts3)),
-        "classify_us": cold_us(lambda: binding.classify(numer, n_end, 0.1, stage, counts)),
-        "update_indexed_us": cold_us(lambda: binding.calib_update_indexed(buf, n_end, news[0], index, ws)),
-        "note": "L2 flushed by a 512 MB write before each call; one call between two events",
-    }
-    del scrub
-    rank_bytes = 12.0 * Nc + 4.0 * n_end
-    cls_bytes = 5.0 * Nc
-    fused_bytes = rank_bytes + len(cfg["alphas"]) * Nc
-    out = {
-        "workload": f"conformal-only stress: Nc={Nc}, n {n0}->{cap}, k={k}, {steps} steps, alphas {list(cfg['alphas'])}",
-        "step": "atts_rank_classify_indexed (3 alphas, one launch) + atts_calib_update_indexed",
-        "pvalues_per_s": Nc * steps / (ms_seq * 1e-3),
-        "ms_sequence": ms_seq, "ms_sequence_eager_launches": min(eager),
-        "ms_sequence_without_index": ms_seq_plain, "pvalues_per_s_without_index": Nc * steps / (ms_seq_plain * 1e-3),
-        "timing": "64-step sequence captured in one CUDA graph, events around the replay, best of 5; working set "
-                  "(<= 14 MB) is L2-resident, so GB/s are algorithmic bytes over time, not DRAM traffic",
-        "rank_us": ms_rank * 1e3, "rank_gbs": rank_bytes / (ms_rank * 1e-3) / 1e9,
-        "rank_frac_hbm": rank_bytes / (ms_rank * 1e-3) / 1e9 / peaks["hbm_gbs"],
-        "classify_us": ms_cls * 1e3, "classify_gbs": cls_bytes / (ms_cls * 1e-3) / 1e9,
-        "update_us": ms_upd * 1e3,
-        "rank_classify_fused_us": ms_fused * 1e3, "rank_classify_fused_gbs": fused_bytes / (ms_fused * 1e-3) / 1e9,
-        "rank_classify_indexed_us": ms_fused_ix * 1e3, "rank_classify_indexed_gbs": fused_bytes / (ms_fused_ix * 1e-3) / 1e9,
-        "update_indexed_us": ms_upd_ix * 1e3,
-        "cold_l2": cold,
-    }
-    if binding.last_device_status() != 0:
-        raise RuntimeError("a conformal kernel reported a device-side error during the benchmark")
-    del scores, numer, p, stage, stage3
-    out.update(conformal_scaled(torch, binding, peaks, graph_ms))
-    return out
 
 
 def make_graph_timer(torch):
@@ -319,16 +239,182 @@ def make_graph_timer(torch):
     return graph_ms
 
 
+def update_bytes(n: int, k: int) -> float:
+    """Algorithmic bytes of one merge-insert: the old buffer read and the merged buffer written once, the new
+    scores read once."""
+    return 8.0 * (n + k) + 4.0 * k
+
+
+def conformal_stress(torch, binding, peaks):
+    """Extra figures on the conformal-only workload: 2^20 candidates against a buffer growing from 65,536 by 4,096 a
+    step, three alphas; kernel times by CUDA events (the working set is L2-resident)."""
+    cfg = inputs.CONFORMAL_STRESS
+    Nc, n0, k, steps = cfg["Nc"], cfg["n0"], cfg["k"], cfg["steps"]
+    alphas = cfg["alphas"]
+    dev = "cuda"
+    hbm = peaks["hbm_gbs"]
+    scores = torch.from_numpy(inputs.lognormal_scores(inputs.BASE_SEED + 1, Nc)).to(dev)
+    calib0 = torch.from_numpy(np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, n0))).to(dev)
+    news = [torch.from_numpy(inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, k)).to(dev) for t in range(steps)]
+    cap = n0 + k * steps
+    buf = torch.empty(cap, device=dev)
+    numer = torch.empty(Nc, dtype=torch.int32, device=dev)
+    p = torch.empty(Nc, device=dev)
+    stage = torch.empty(Nc, dtype=torch.uint8, device=dev)
+    counts = torch.empty(3, dtype=torch.int32, device=dev)
+    stage3 = torch.empty((len(alphas), Nc), dtype=torch.uint8, device=dev)
+    counts3 = torch.empty((len(alphas), 3), dtype=torch.int32, device=dev)
+    ws = torch.empty(binding.calib_workspace_bytes(cap, k), dtype=torch.uint8, device=dev)
+    index = torch.empty(binding.calib_index_bytes(cap), dtype=torch.uint8, device=dev)
+    side = torch.cuda.Stream()
+
+    def sequence_plain():
+        buf[:n0] = calib0
+        n = n0
+        for t in range(steps):
+            binding.rank_classify(scores, buf, n, alphas, numer, p, stage3, counts3)
+            n = binding.calib_update(buf, n, news[t], ws)
+        return n
+
+    def sequence():
+        # the calibration state is the buffer and its index; every update leaves both describing the new fill
+        buf[:n0] = calib0
+        binding.calib_index_build(buf, n0, index)
+        n = n0
+        for t in range(steps):
+            binding.rank_classify_indexed(scores, buf, n, index, alphas, numer, p, stage3, counts3)
+            n = binding.calib_update_indexed(buf, n, news[t], index, ws)
+        return n
+
+    def sequence_two_streams():
+        # the update of step t needs nothing the rank of step t writes: it runs on a second stream beside it; the
+        # next rank waits for the update, the next update for this rank (it overwrites what this rank reads)
+        main = torch.cuda.current_stream()
+        buf[:n0] = calib0
+        binding.calib_index_build(buf, n0, index)
+        n = n0
+        for t in range(steps):
+            side.wait_stream(main)
+            binding.rank_classify_indexed(scores, buf, n, index, alphas, numer, p, stage3, counts3)
+            with torch.cuda.stream(side):
+                n = binding.calib_update_indexed(buf, n, news[t], index, ws)
+            main.wait_stream(side)
+        return n
+
+    graph_ms = make_graph_timer(torch)
+    ms_seq_plain = graph_ms(sequence_plain)
+    ms_seq = graph_ms(sequence)
+    ms_seq2 = graph_ms(sequence_two_streams)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    eager = []
+    for _ in range(3):
+        e0.record()
+        sequence()
+        e1.record()
+        torch.cuda.synchronize()
+        eager.append(e0.elapsed_time(e1))
+
+    # ---- single calls at the last step's sizes.  The update is timed together with a copy that restores the buffer
+    # (repeated inserts into the same buffer would drift its contents), and that copy alone is subtracted.
+    n_end = cap - k
+    calib_end = torch.sort(torch.cat([calib0] + news[:-1])).values.contiguous()
+    assert calib_end.numel() == n_end
+
+    def restore():
+        buf[:n_end] = calib_end
+
+    restore()
+    ms_restore = graph_ms(restore, reps=20)
+    ms_rank = graph_ms(lambda: binding.conformal_rank(scores, buf, n_end, numer, p), reps=20)
+    ms_cls = graph_ms(lambda: binding.classify(numer, n_end, 0.1, stage, counts), reps=20)
+    ms_fused = graph_ms(lambda: binding.rank_classify(scores, buf, n_end, alphas, numer, p, stage3, counts3), reps=20)
+
+    def upd_plain():
+        restore()
+        binding.calib_update(buf, n_end, news[-1], ws)
+
+    ms_upd = graph_ms(upd_plain, reps=20) - ms_restore
+    restore()
+    binding.calib_index_build(buf, n_end, index)
+    ms_fused_ix = graph_ms(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, alphas, numer, p, stage3,
+                                                                 counts3), reps=20)
+    # the indexed update reads the index's copy of fill n_end, which repeated calls leave as it is
+    ms_upd_ix = graph_ms(lambda: binding.calib_update_indexed(buf, n_end, news[-1], index, ws), reps=20)
+    # a drifted batch: every new score above the buffer's largest entry (one block owns and sorts them all)
+    drift = (news[-1] + calib_end[-1]).contiguous()
+    ms_upd_ix_drift = graph_ms(lambda: binding.calib_update_indexed(buf, n_end, drift, index, ws), reps=20)
+    # The same calls with a cold L2: 512 MB are written between repetitions, one call is timed by events (the events'
+    # own few microseconds are inside), median of 9.
+    scrub = torch.empty(128 << 20, dtype=torch.float32, device=dev)
+
+    def cold_us(fn):
+        ts = []
+        for _ in range(9):
+            scrub.fill_(1.0)
+            torch.cuda.synchronize()
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+
+    restore()
+    cold = {
+        "rank_classify_indexed_us": cold_us(lambda: binding.rank_classify_indexed(scores, buf, n_end, index, alphas,
+                                                                              numer, p, stage3, counts3)),
+        "rank_classify_us": cold_us(lambda: binding.rank_classify(scores, buf, n_end, alphas, numer, p, stage3, counts3)),
+        "classify_us": cold_us(lambda: binding.classify(numer, n_end, 0.1, stage, counts)),
+        "update_indexed_us": cold_us(lambda: binding.calib_update_indexed(buf, n_end, news[-1], index, ws)),
+        "note": "L2 flushed by a 512 MB write before each call; one call between two events",
+    }
+    del scrub
+    rank_bytes = 12.0 * Nc + 4.0 * n_end
+    cls_bytes = 5.0 * Nc
+    fused_bytes = rank_bytes + len(alphas) * Nc
+    # algorithmic bytes of the whole 64-step sequence: per step the rank + three alphas in one pass and one merge-insert
+    seq_bytes = sum(12.0 * Nc + len(alphas) * Nc + 4.0 * (n0 + k * t) + update_bytes(n0 + k * t, k) for t in range(steps))
+    out = {
+        "workload": f"conformal-only stress: Nc={Nc}, n {n0}->{cap}, k={k}, {steps} steps, alphas {list(alphas)}",
+        "step": "atts_rank_classify_indexed (3 alphas, one launch) + atts_calib_update_indexed (one launch)",
+        "pvalues_per_s": Nc * steps / (ms_seq * 1e-3),
+        "ms_sequence": ms_seq, "us_per_step": ms_seq * 1e3 / steps, "ms_sequence_eager_launches": min(eager),
+        "sequence_algorithmic_gbs": seq_bytes / (ms_seq * 1e-3) / 1e9,
+        "sequence_frac_hbm": seq_bytes / (ms_seq * 1e-3) / 1e9 / hbm,
+        "ms_sequence_two_streams": ms_seq2, "pvalues_per_s_two_streams": Nc * steps / (ms_seq2 * 1e-3),
+        "ms_sequence_without_index": ms_seq_plain, "pvalues_per_s_without_index": Nc * steps / (ms_seq_plain * 1e-3),
+        "timing": "64-step sequence captured in one CUDA graph, events around the replay, best of 5; working set "
+                  "(<= 14 MB) is L2-resident, so GB/s are algorithmic bytes over time, not DRAM traffic; "
+                  "two_streams: each update on a second stream beside the rank of the same fill",
+        "rank_us": ms_rank * 1e3, "rank_gbs": rank_bytes / (ms_rank * 1e-3) / 1e9,
+        "rank_frac_hbm": rank_bytes / (ms_rank * 1e-3) / 1e9 / hbm,
+        "classify_us": ms_cls * 1e3, "classify_gbs": cls_bytes / (ms_cls * 1e-3) / 1e9,
+        "update_us": ms_upd * 1e3, "update_gbs": update_bytes(n_end, k) / (ms_upd * 1e-3) / 1e9,
+        "rank_classify_fused_us": ms_fused * 1e3, "rank_classify_fused_gbs": fused_bytes / (ms_fused * 1e-3) / 1e9,
+        "rank_classify_indexed_us": ms_fused_ix * 1e3, "rank_classify_indexed_gbs": fused_bytes / (ms_fused_ix * 1e-3) / 1e9,
+        "update_indexed_us": ms_upd_ix * 1e3, "update_indexed_gbs": update_bytes(n_end, k) / (ms_upd_ix * 1e-3) / 1e9,
+        "update_indexed_drifted_batch_us": ms_upd_ix_drift * 1e3,
+        "update_bytes": "8 (n + k) + 4 k per merge-insert (the old buffer read, the merged buffer written, the new scores read)",
+        "cold_l2": cold,
+    }
+    if binding.last_device_status() != 0:
+        raise RuntimeError("a conformal kernel reported a device-side error during the benchmark")
+    del scores, numer, p, stage, stage3
+    out.update(conformal_scaled(torch, binding, peaks, graph_ms))
+    return out
+
+
 def conformal_scaled(torch, binding, peaks, graph_ms):
     """The conformal kernels at sizes where HBM is the limit (extra points beside the five workload shapes)."""
     dev = "cuda"
     out = {}
+    hbm = peaks["hbm_gbs"]
     k = inputs.CONFORMAL_STRESS["k"]
     counts = torch.empty(3, dtype=torch.int32, device=dev)
     new0 = torch.from_numpy(inputs.lognormal_scores(inputs.BASE_SEED + 3, k)).to(dev)
-    # The same kernels where HBM is the limit: 2^26 candidates (805 MB of traffic per rank pass) against the
-    # model-sized buffer n = 4096, and a merge-insert into a 2^22-entry buffer.
-    big, n_small = 1 << 26, 4096
+    # 2^26 candidates (805 MB of traffic per rank pass) against the model-sized buffer n = 4096 and against a
+    # buffer of 2^22 entries, and a merge-insert into a 2^22-entry buffer.
+    big, n_small, n_big = 1 << 26, 4096, 1 << 22
     gen = torch.Generator(device=dev)
     gen.manual_seed(inputs.BASE_SEED + 7)
     sc = torch.randn(big, device=dev, generator=gen).exp_()
@@ -336,17 +422,32 @@ def conformal_scaled(torch, binding, peaks, graph_ms):
     nm = torch.empty(big, dtype=torch.int32, device=dev)
     pv = torch.empty(big, device=dev)
     st = torch.empty(big, dtype=torch.uint8, device=dev)
+
+    def point(ms, nbytes, **extra):
+        d = {"us": ms * 1e3, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_hbm": nbytes / (ms * 1e-3) / 1e9 / hbm}
+        d.update(extra)
+        return d
+
     ms = graph_ms(lambda: binding.conformal_rank(sc, cal, n_small, nm, pv), reps=2)
-    out["scaled_rank"] = {"Nc": big, "n": n_small, "us": ms * 1e3, "gbs": 12.0 * big / (ms * 1e-3) / 1e9,
-                          "frac_hbm": 12.0 * big / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["scaled_rank"] = point(ms, 12.0 * big, Nc=big, n=n_small)
+    # the same candidates against 2^22 calibration scores: with the index (three 32-byte loads per candidate from the
+    # L2-resident index, bound by the rate at which an SM serves divergent loads) and without it
+    bufb = torch.empty(n_big + k, device=dev)
+    bufb[:n_big] = torch.sort(torch.randn(n_big, device=dev, generator=gen).exp_()).values
+    calib_big = bufb[:n_big].clone()
+    ixb = torch.empty(binding.calib_index_bytes(n_big + k), dtype=torch.uint8, device=dev)
+    binding.calib_index_build(bufb, n_big, ixb)
+    ms = graph_ms(lambda: binding.rank_classify_indexed(sc, bufb, n_big, ixb, (), nm, pv), reps=2)
+    out["scaled_rank_large_buffer_indexed"] = point(ms, 12.0 * big + 4.0 * n_big, Nc=big, n=n_big)
+    ms = graph_ms(lambda: binding.conformal_rank(sc, bufb, n_big, nm, pv), reps=1)
+    out["scaled_rank_large_buffer_without_index"] = point(ms, 12.0 * big + 4.0 * n_big, Nc=big, n=n_big)
+    binding.conformal_rank(sc, cal, n_small, nm, pv)
     ms = graph_ms(lambda: binding.classify(nm, n_small, 0.1, st, counts), reps=2)
-    out["scaled_classify"] = {"Nc": big, "us": ms * 1e3, "gbs": 5.0 * big / (ms * 1e-3) / 1e9,
-                              "frac_hbm": 5.0 * big / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["scaled_classify"] = point(ms, 5.0 * big, Nc=big)
     tau = torch.empty(1, device=dev)
     binding.threshold(cal, n_small, 0.1, tau)
     ms = graph_ms(lambda: binding.classify_threshold(sc, tau, st, counts), reps=2)
-    out["scaled_classify_threshold"] = {"Nc": big, "us": ms * 1e3, "gbs": 5.0 * big / (ms * 1e-3) / 1e9,
-                                        "frac_hbm": 5.0 * big / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["scaled_classify_threshold"] = point(ms, 5.0 * big, Nc=big)
     # budget report: positions of the stage-3 samples among 2^26 (stages from the classify call above, alpha = 0.1)
     ids = torch.empty(big // 4, dtype=torch.int32, device=dev)
     cnt = torch.empty(1, dtype=torch.int32, device=dev)
@@ -354,10 +455,8 @@ def conformal_scaled(torch, binding, peaks, graph_ms):
     binding.classify(nm, n_small, 0.1, st, counts)
     ms = graph_ms(lambda: binding.takeover_ids(st, ids, cnt, ws_ids), reps=2)
     B = int(cnt.cpu().numpy().view(np.uint32)[0])
-    ids_bytes = 1.0 * big + 4.0 * B      # every stage byte once, every position once
-    out["scaled_takeover_ids"] = {"Nc": big, "B": B, "us": ms * 1e3, "gbs": ids_bytes / (ms * 1e-3) / 1e9,
-                                  "frac_hbm": ids_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                  "note": "three launches; the stage bytes are read twice (count, then write)"}
+    out["scaled_takeover_ids"] = point(ms, 1.0 * big + 4.0 * B, Nc=big, B=B,
+                                       note="one pass: every stage byte read once, every position written once")
     del ids, ws_ids
     # conditional coverage: 2^24 candidates, each ranked against its own input's 64 calibration scores
     ncond, G, m = 1 << 24, 1 << 16, 64
@@ -367,25 +466,117 @@ def conformal_scaled(torch, binding, peaks, graph_ms):
     dn = torch.empty(ncond, dtype=torch.int32, device=dev)
     ms = graph_ms(lambda: binding.conformal_rank_conditional(sc[:ncond], gid, segs, seg_off, nm[:ncond], dn, pv[:ncond]), reps=2)
     cbytes = 20.0 * ncond    # score + group id in, numer + denom + p out
-    out["scaled_rank_conditional"] = {"Nc": ncond, "groups": G, "group_size": m, "us": ms * 1e3,
-                                      "gbs": cbytes / (ms * 1e-3) / 1e9, "frac_hbm": cbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    out["scaled_rank_conditional"] = point(ms, cbytes, Nc=ncond, groups=G, group_size=m)
     # the same with the candidates of one input adjacent (how a batch of per-input samples arrives)
     gid_grouped = torch.sort(gid).values
     ms = graph_ms(lambda: binding.conformal_rank_conditional(sc[:ncond], gid_grouped, segs, seg_off, nm[:ncond], dn, pv[:ncond]), reps=2)
-    out["scaled_rank_conditional_grouped"] = {"Nc": ncond, "groups": G, "group_size": m, "us": ms * 1e3,
-                                              "gbs": cbytes / (ms * 1e-3) / 1e9, "frac_hbm": cbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                              "note": "group ids non-decreasing: candidates of one input are adjacent"}
+    out["scaled_rank_conditional_grouped"] = point(ms, cbytes, Nc=ncond, groups=G, group_size=m,
+                                                   note="group ids non-decreasing: candidates of one input are adjacent")
     del sc, nm, pv, st, gid, gid_grouped, dn, segs
-    n_big = 1 << 22
-    bufb = torch.empty(n_big + k, device=dev)
-    bufb[:n_big] = torch.sort(torch.randn(n_big, device=dev, generator=gen).exp_()).values
+    # merge-insert of 4096 scores into 2^22: the call without an index (merge into the workspace + copy back, timed
+    # with a restoring copy that is subtracted) and the indexed call (one pass, no copy back)
     wsb = torch.empty(binding.calib_workspace_bytes(n_big, k), dtype=torch.uint8, device=dev)
-    ms = graph_ms(lambda: binding.calib_update(bufb, n_big, new0, wsb), reps=2)
-    upd_bytes = 16.0 * (n_big + k)   # merge: read + write; copy back: read + write
-    out["scaled_update"] = {"n": n_big, "k": k, "us": ms * 1e3, "gbs": upd_bytes / (ms * 1e-3) / 1e9,
-                            "frac_hbm": upd_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                            "bytes": "16 per element: merge into the workspace and copy back"}
+
+    def restore():
+        bufb[:n_big] = calib_big
+
+    ms_restore = graph_ms(restore, reps=4)
+
+    def upd_plain():
+        restore()
+        binding.calib_update(bufb, n_big, new0, wsb)
+
+    ms = graph_ms(upd_plain, reps=4) - ms_restore
+    out["scaled_update"] = point(ms, update_bytes(n_big, k), n=n_big, k=k,
+                                 note="merge into the workspace, then a copy back: the implementation moves 16 (n + k) bytes")
+    restore()
+    binding.calib_index_build(bufb, n_big, ixb)
+    ms = graph_ms(lambda: binding.calib_update_indexed(bufb, n_big, new0, ixb, wsb), reps=4)
+    out["scaled_update_indexed"] = point(ms, update_bytes(n_big, k), n=n_big, k=k,
+                                         note="one pass from one half of the index into the other half and the buffer: "
+                                              "the implementation moves 12 (n + k) bytes")
+    out["bytes"] = "algorithmic: rank 12 Nc (+ 4 n), classify 5 Nc, budget report Nc + 4 B, merge-insert 8 (n + k) + 4 k"
     return out
+
+
+def per_config_leg(torch, binding, peaks, name, dev, target_ms=1000.0):
+    """One of the other workload shapes, timed like the bench line's device-resident leg: step = score + rank +
+    classify at each of the shape's alphas + calibration update.  The inputs have the recipe's distributions but are
+    drawn on the device (torch Philox) to keep the whole benchmark within minutes."""
+    c = inputs.CONFIGS[name]
+    N, T, d, V, n0, alphas = c["N"], c["T"], c["d"], c["V"], c["n"], c["alphas"]
+    M = N * T
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(inputs.BASE_SEED + 200 + sorted(inputs.CONFIGS).index(name))
+    W_d = torch.empty(V, d, dtype=torch.bfloat16, device=dev)
+    for r0 in range(0, V, 16384):
+        r1 = min(r0 + 16384, V)
+        W_d[r0:r1] = (torch.randn(r1 - r0, d, device=dev, generator=gen) * 0.02).to(torch.bfloat16)
+    cdf = torch.cumsum(torch.arange(1, V + 1, device=dev, dtype=torch.float64) ** -1.1, 0)
+    cdf /= cdf[-1].clone()
+    off_d = torch.from_numpy(inputs.seg_offsets(N, T)).to(dev)
+
+    def draw_batch(H):
+        for r0 in range(0, M, 8192):
+            x = torch.randn(min(8192, M - r0), d, device=dev, generator=gen)
+            H[r0:r0 + x.shape[0]] = (x / x.pow(2).mean(1, keepdim=True).sqrt()).to(torch.bfloat16)
+        u = torch.rand(M, device=dev, dtype=torch.float64, generator=gen)
+        return torch.searchsorted(cdf, u, right=True).clamp_(max=V - 1).to(torch.int32)
+
+    H_d = torch.empty(M, d, dtype=torch.bfloat16, device=dev)
+    score_d = torch.empty(N, device=dev)
+    numer = torch.empty(N, dtype=torch.int32, device=dev)
+    pval = torch.empty(N, device=dev)
+    stage = torch.empty(N, dtype=torch.uint8, device=dev)
+    counts = torch.empty(3, dtype=torch.int32, device=dev)
+    ws_s = torch.empty(binding.score_workspace_bytes(M, d, V, N), dtype=torch.uint8, device=dev)
+    cap = n0 + N * 2100
+    calib = torch.empty(cap, device=dev)
+    ws_c = torch.empty(binding.calib_workspace_bytes(cap, N), dtype=torch.uint8, device=dev)
+    n = 0
+    for _ in range(n0 // N):       # calibration buffer: n0 scores of calibration batches through the same calls
+        ids_c = draw_batch(H_d)
+        binding.score_logprob(H_d, W_d, ids_c, off_d, None, score_d, ws_s)
+        n = binding.calib_update(calib, n, score_d, ws_c)
+    ids_d = draw_batch(H_d)
+    state = {"n": n}
+
+    def step():
+        binding.score_logprob(H_d, W_d, ids_d, off_d, None, score_d, ws_s)
+        binding.conformal_rank(score_d, calib, state["n"], numer, pval)
+        for alpha in alphas:
+            binding.classify(numer, state["n"], alpha, stage, counts)
+        state["n"] = binding.calib_update(calib, state["n"], score_d, ws_c)
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    est = e0.elapsed_time(e1) / 3
+    K = int(min(2000, max(10, target_ms / max(est, 1e-3))))
+    binding.profile_begin(K)
+    e0.record()
+    for _ in range(K):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    k1 = binding.profile_end()
+    ms = e0.elapsed_time(e1) / K
+    if binding.last_device_status() != 0:
+        raise RuntimeError(f"device status set while timing the {name} shape")
+    k1_ms = sum(k1) / len(k1)
+    tflops = 2.0 * M * d * V / (k1_ms * 1e-3) / 1e12
+    return {"workload": f"N={N} x T={T}, d={d}, V={V}, n={n0}, alphas {list(alphas)}", "steps": K, "ms_per_step": ms,
+            "tokens_per_s": M / (ms * 1e-3), "fused_kernel_ms": k1_ms, "fused_kernel_tflops": tflops,
+            "frac_of_sustained_peak": tflops / peaks["bf16_tflops_sustained"], "frac_of_burst_peak": tflops / peaks["bf16_tflops"],
+            "data": "synthetic, drawn on the device with the recipe's distributions",
+            "l2": "inputs larger than L2" if (V * d * 2 + M * d * 2) > (126 << 20) else
+                  "inputs fit in L2 (W %.1f MB + H %.1f MB): warm-cache figure" % (V * d * 2 / 1e6, M * d * 2 / 1e6)}
 
 
 def run_ours(args):
@@ -655,7 +846,10 @@ def run_ours(args):
                      "frac": achieved / peaks["bf16_tflops_sustained"], "peak_kind": f"{peak_kind}, sustained bf16 GEMM "
                      "(kernel timed inside a long step)", "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
                      "kernel_ms": k1_avg, "flops_per_launch": flops,
-                     "traffic": k1_traffic_bytes() if args.workload == WORKLOAD else None},
+                     "traffic": k1_traffic_bytes() if args.workload == WORKLOAD else None,
+                     "traffic_note": "stored figure: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of "
+                                     "this kernel source on this workload (mean of 3 launches), not measured in this run; "
+                                     "captures on other boxes ranged 45-98 GB per launch; null once the kernel source changes"},
         "stage_counts_last_step": stage_counts_last, "calib_n_end": state["n"],
     }
     # Asynchronous arithmetic intensity of the step (the paper's r = T_c / (T_m + T_s)): T_c the fused kernel's time,
@@ -676,18 +870,27 @@ def run_ours(args):
     if rank == 0 and world == 1:
         if not args.no_cpu_baseline:
             from oracle import atts_oracle as orc
-            rows = args.oracle_rows
+            # one whole draft sample plus token rows scattered over the rest of the batch
+            whole = 1 if args.oracle_rows >= 256 else 0
+            plan = oracle_rows_plan(M, T, whole, args.oracle_rows, inputs.BASE_SEED + 9)
             cal = calib[:state["n"]].cpu().numpy()
+            ids_np = ids_host.numpy()
+            rest = score_d.cpu().numpy()[whole:]        # the other samples' scores feed the conformal steps
             t0 = time.perf_counter()
-            oracle_step(orc, Hb, Wb, ids_host.numpy(), rows, N, cal, ALPHA)
+            oracle_step(orc, Hb[plan], Wb, ids_np[plan], whole * T, T, rest, cal, ALPHA)
             dt = time.perf_counter() - t0
-            line["cpu_baseline"] = {"value": rows / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-                                    "sample": f"{rows} of {M} token rows of the same batch (full d and V) in {dt:.1f} s, "
-                                              f"then rank/classify/update on N={N} scores"}
+            line["cpu_baseline"] = {"value": plan.size / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                    "sample": f"{plan.size} of {M} token rows of the same batch (full d and V) in {dt:.1f} s: "
+                                              f"{whole} whole sample(s) of {T} tokens plus {plan.size - whole * T} rows scattered "
+                                              f"over the rest by a seeded permutation; then rank/classify/update on N={N} scores"}
             line["cpu_baseline"]["conformal_only"] = oracle_conformal_steps(orc)
-        if not args.no_conformal:
-            del H_d, W_d
+        del H_d, W_d, bufs
+        torch.cuda.empty_cache()
+        if not args.no_per_config and args.workload == WORKLOAD:
+            line["per_config"] = {name: per_config_leg(torch, binding, peaks, name, dev)
+                                  for name in ("tiny", "7b", "70b")}
             torch.cuda.empty_cache()
+        if not args.no_conformal:
             line["conformal_stress"] = conformal_stress(torch, binding, peaks)
     if rank == 0:
         print(json.dumps(line), flush=True)
@@ -706,6 +909,7 @@ def main():
                     help="shape to run (default: the bench line's workload; others are for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-conformal", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the tiny / 7B / 70B shapes beside the bench line")
     ap.add_argument("--no-library-gemm", action="store_true", help="skip the torch.matmul comparison on the same GPU")
     ap.add_argument("--conformal-scaled-only", action="store_true",
                     help="run only the HBM-scale points of the conformal kernels (for profiling)")

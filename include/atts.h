@@ -370,6 +370,23 @@ int atts_debug_score_unit(int64_t M, int64_t d, int64_t V, int32_t workers, int3
                           int32_t* out);
 
 /*
+ * Bounded waits of the scoring kernel (diagnostic; the paper has no counterpart).  Every wait inside
+ * atts_score_logprob's fused kernel (for a shared-memory stage to fill or drain, for an accumulator to complete or be
+ * read) gives up after a number of SM cycles; the kernel then stops, lets copies in flight land, frees its tensor
+ * memory and returns, ATTS_DEV_WAIT_EXPIRED is recorded and atts_last_device_status returns ATTS_ERR_TIMEOUT.  The
+ * outputs of such a call are invalid; the context stays usable.
+ *   atts_debug_set_wait   limit_cycles > 0: the bound for later calls in this process (default 4e9, about two seconds;
+ *                         the environment variable ATTS_WAIT_LIMIT presets it); limit_cycles <= 0: the default.
+ *                         withhold_loads = 1: the kernel's producer issues no loads at all, so the first wait for data
+ *                         can never be satisfied and must run out - the way to exercise the expiry path without a
+ *                         fault (nothing is in flight when the kernel gives up); 0: normal operation.
+ *   atts_debug_score_form host out *ctas: 1 if atts_score_logprob would run M x d x V on single CTAs on the current
+ *                         device, 2 if on CTA pairs.
+ */
+int atts_debug_set_wait(int64_t limit_cycles, int32_t withhold_loads);
+int atts_debug_score_form(int64_t M, int64_t d, int64_t V, int32_t* ctas);
+
+/*
  * Timing hooks (measurement aid; the paper has no counterpart).  Between atts_profile_begin and
  * atts_profile_end every atts_score_logprob call records a pair of CUDA events on its stream
  * directly around the fused LM-head kernel, for at most `max_records` calls (<= 4096).

@@ -21,7 +21,7 @@ EXPORTS = (
     "atts_threshold", "atts_classify_threshold", "atts_conformal_rank_conditional", "atts_classify_conditional",
     "atts_debug_score_plan", "atts_debug_score_unit", "atts_score_slice", "atts_score_combine",
     "atts_calib_index_bytes", "atts_calib_index_build", "atts_calib_update_indexed", "atts_rank_classify_indexed",
-    "atts_takeover_ids_workspace_bytes", "atts_takeover_ids",
+    "atts_takeover_ids_workspace_bytes", "atts_takeover_ids", "atts_debug_set_wait", "atts_debug_score_form",
 )
 
 STAGE_DRAFT, STAGE_ACCEPTED, STAGE_TARGET = 1, 2, 3
@@ -86,6 +86,8 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
                                                c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.atts_takeover_ids_workspace_bytes.argtypes = [c_int64, POINTER(c_size_t)]
     lib.atts_takeover_ids.argtypes = [c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.atts_debug_set_wait.argtypes = [c_int64, c_int32]
+    lib.atts_debug_score_form.argtypes = [c_int64, c_int64, c_int64, POINTER(c_int32)]
     lib.atts_profile_begin.argtypes = [c_int]
     lib.atts_profile_end.argtypes = [POINTER(ctypes.c_float), c_int, POINTER(c_int)]
     for name in EXPORTS[2:]:
@@ -301,6 +303,19 @@ def last_device_status() -> int:
     if st != 0:
         raise AttsError(st, "atts_last_device_status")
     return bits.value
+
+
+def debug_set_wait(limit_cycles: int = 0, withhold_loads: bool = False) -> None:
+    """Bound (SM cycles; <= 0 restores the default) of the scoring kernel's pipeline waits for later calls, and the
+    diagnostic switch that makes its producer issue no loads so that the first wait for data runs out."""
+    _check(load().atts_debug_set_wait(int(limit_cycles), 1 if withhold_loads else 0), "atts_debug_set_wait")
+
+
+def debug_score_form(M: int, d: int, V: int) -> int:
+    """1 if score_logprob runs this shape on single CTAs on the current device, 2 if on CTA pairs."""
+    out = c_int32(0)
+    _check(load().atts_debug_score_form(M, d, V, ctypes.byref(out)), "atts_debug_score_form")
+    return out.value
 
 
 def profile_begin(max_records: int = 1024) -> None:

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <cudaTypedefs.h>
 #include <math.h>
+#include <stdlib.h>
+#include <atomic>
 #include <mutex>
 
 #include "conformal.cuh"
@@ -26,6 +28,23 @@ struct DeviceInfo {
 
 static DeviceInfo g_info[64];
 static std::mutex g_mu;
+
+// Bound of the scoring kernel's pipeline waits, in SM cycles, and the diagnostic switch that makes the first wait
+// run out (atts_debug_set_wait).  The environment variable ATTS_WAIT_LIMIT, read once, presets the bound.
+static std::atomic<long long> g_wait_limit{0};   // 0: not set yet
+static std::atomic<int> g_withhold_loads{0};
+static long long wait_limit() {
+  long long v = g_wait_limit.load(std::memory_order_relaxed);
+  if (v == 0) {
+    v = kWaitLimitCycles;
+    if (const char* e = getenv("ATTS_WAIT_LIMIT")) {
+      const long long x = atoll(e);
+      if (x > 0) v = x;
+    }
+    g_wait_limit.store(v, std::memory_order_relaxed);
+  }
+  return v;
+}
 
 // Probes the current device once: architecture, SM count, address of the status word, driver entry
 // point for tensor-map encoding, and the opt-in shared-memory sizes of the kernels.
@@ -274,6 +293,8 @@ static int score_impl(const void* hidden_bf16, const void* lm_head_bf16, const i
   if (st != ATTS_OK) return st;
   ScorePlan plan = choose_score_plan(di, M, d, V);
   plan.vocab_offset = (int)vocab_offset;
+  plan.wait_limit = wait_limit();
+  plan.withhold_loads = g_withhold_loads.load(std::memory_order_relaxed);
   const ScoreWs ws = score_ws(plan);
   if (workspace_bytes < ws.total) return ATTS_ERR_WORKSPACE;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -552,11 +573,12 @@ int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, u
   return launch_status();
 }
 
-// Workspace of atts_takeover_ids: [one 64-bit word per tile][ticket counter], cleared before the launch.
+// Workspace of atts_takeover_ids: [one 64-bit word per range][ticket counter], cleared before the launch.  A range
+// is at least 4096 stage bytes, which bounds the number of ranges whatever the device.
 int atts_takeover_ids_workspace_bytes(int64_t Nc, size_t* bytes) {
   if (!bytes) return ATTS_ERR_NULL;
   if (Nc < 0 || Nc >= (1ll << 31)) return ATTS_ERR_SHAPE;
-  *bytes = round_up((size_t)((Nc + kIdsTile - 1) / kIdsTile) * sizeof(unsigned long long) + 8, 256) + 256;
+  *bytes = round_up((size_t)((Nc + kIdsRowBytes - 1) / kIdsRowBytes) * sizeof(unsigned long long) + 8, 256) + 256;
   return ATTS_OK;
 }
 
@@ -579,16 +601,20 @@ int atts_takeover_ids(const uint8_t* stage, int64_t Nc, int32_t* ids, int64_t id
     }
     return ATTS_OK;
   }
-  const int tiles = (int)((Nc + kIdsTile - 1) / kIdsTile);
+  // about four ranges per SM, a range being Q rows of 4096 bytes (1 <= Q <= 32)
+  const int64_t per_range = (Nc + (int64_t)di->sm_count * 4 - 1) / ((int64_t)di->sm_count * 4);
+  int64_t Q = (per_range + kIdsRowBytes - 1) / kIdsRowBytes;
+  Q = Q < 1 ? 1 : (Q > kIdsMaxRows ? kIdsMaxRows : Q);
+  const int ranges = (int)((Nc + Q * kIdsRowBytes - 1) / (Q * kIdsRowBytes));
   const bool vec = aligned(stage, 16);
   unsigned long long* state = static_cast<unsigned long long*>(workspace);
-  unsigned int* ticket = reinterpret_cast<unsigned int*>(state + tiles);
-  if (tiles > 1 && cudaMemsetAsync(workspace, 0, (size_t)tiles * sizeof(unsigned long long) + 8, stream) != cudaSuccess) {
+  unsigned int* ticket = reinterpret_cast<unsigned int*>(state + ranges);
+  if (ranges > 1 && cudaMemsetAsync(workspace, 0, (size_t)ranges * sizeof(unsigned long long) + 8, stream) != cudaSuccess) {
     cudaGetLastError();
     return ATTS_ERR_CUDA;
   }
-  int blocks = tiles < di->sm_count * 6 ? tiles : di->sm_count * 6;
-  takeover_ids_kernel<<<blocks, kIdsThreads, 0, stream>>>(stage, Nc, tiles, vec, state, ticket, ids, ids_cap, count,
+  const int blocks = ranges < di->sm_count * 8 ? ranges : di->sm_count * 8;
+  takeover_ids_kernel<<<blocks, kIdsThreads, 0, stream>>>(stage, Nc, (int)Q, ranges, vec, state, ticket, ids, ids_cap, count,
                                                          di->dev_status);
   return launch_status();
 }
@@ -869,6 +895,24 @@ int atts_debug_score_unit(int64_t M, int64_t d, int64_t V, int32_t workers, int3
   int rb, c, nt0, nt1;
   decode_unit(p, u, rb, c, nt0, nt1);
   out[0] = rb; out[1] = c; out[2] = nt0; out[3] = nt1;
+  return ATTS_OK;
+}
+
+int atts_debug_score_form(int64_t M, int64_t d, int64_t V, int32_t* ctas) {
+  if (!ctas) return ATTS_ERR_NULL;
+  int st = check_score_shape(M, d, V, 0);
+  if (st != ATTS_OK) return st;
+  const DeviceInfo* di;
+  st = device_info(&di);
+  if (st != ATTS_OK) return st;
+  *ctas = choose_score_plan(di, M, d, V).ctas;
+  return ATTS_OK;
+}
+
+int atts_debug_set_wait(int64_t limit_cycles, int32_t withhold_loads) {
+  if (withhold_loads != 0 && withhold_loads != 1) return ATTS_ERR_ARG;
+  g_wait_limit.store(limit_cycles > 0 ? (long long)limit_cycles : kWaitLimitCycles, std::memory_order_relaxed);
+  g_withhold_loads.store(withhold_loads, std::memory_order_relaxed);
   return ATTS_OK;
 }
 

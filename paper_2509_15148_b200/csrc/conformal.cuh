@@ -791,83 +791,65 @@ classify_kernel(const uint32_t* __restrict__ numer, int64_t Nc, uint32_t k_alpha
 constexpr int kSortMaxK = 16384;          // new keys per launch (larger batches are inserted slice by slice)
 constexpr int kMergeThreads = 1024;
 constexpr int kMergeTileMax = 8192;       // old entries per tile (32 KB of shared memory)
-constexpr int kMergeRankSortMax = 384;    // own keys up to this many are sorted by all-pairs ranking, more by a radix sort
+constexpr int kMergeRankSortMax = 384;    // own keys up to this many are sorted by all-pairs ranking, more by a bitonic network
 
-constexpr int kRadixHistStride = 33;      // one column per warp, padded against bank conflicts
-
-// Block-wide radix sort (least significant byte first, four passes) of a[0, m), m <= 16384, by the kMergeThreads
-// threads of a block; b is a second array of the same size, both hold at least m rounded up to a multiple of
-// kMergeThreads words.  The sorted keys end in a.  hist: 256 * kRadixHistStride words, wsum: 32 words (shared).
-// Warp w owns the 32 E consecutive keys from w * 32 E on (E = keys per thread); in each pass a key's destination is
-// the number of keys with a smaller digit, plus those with the same digit in earlier warps, plus those with the
-// same digit earlier in its own warp, which keeps every pass stable.
-__device__ __forceinline__ void block_radix_sort(uint32_t* a, uint32_t* b, int m, uint32_t* hist, uint32_t* wsum) {
-  const int E = (m + kMergeThreads - 1) / kMergeThreads;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int i = m + threadIdx.x; i < E * kMergeThreads; i += kMergeThreads) a[i] = 0xFFFFFFFFu;   // sorts last
-  uint32_t* src = a;
-  uint32_t* dst = b;
-  const int entries = 256 * kRadixHistStride;
-  constexpr int kPer = (256 * kRadixHistStride + kMergeThreads - 1) / kMergeThreads;   // histogram words per thread in the scan
-  for (int shift = 0; shift < 32; shift += 8) {
-    for (int i = threadIdx.x; i < entries; i += kMergeThreads) hist[i] = 0u;
-    __syncthreads();
-    const uint32_t* mine = src + warp * 32 * E + lane;
-    uint32_t offs[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // two 16-bit offsets per word
+// Block-wide bitonic sort, ascending, of the kMergeThreads * E keys in a[] (shared memory; the caller pads with a key
+// above all others).  Thread t holds keys t E .. t E + E - 1 in registers: a compare-exchange whose partner lies in
+// the same thread is done in registers, one whose partner lies in the same warp by a shuffle, and only the ones
+// across warps go through shared memory - 15 of the 78 steps for 4096 keys.
+template <int E>
+__device__ __forceinline__ void block_bitonic_sort(uint32_t* a) {
+  constexpr int kLogE = E == 1 ? 0 : E == 2 ? 1 : E == 4 ? 2 : E == 8 ? 3 : 4;
+  const int base = threadIdx.x * E;
+  uint32_t v[E];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      if (j < E) {
-        const uint32_t d = (mine[32 * j] >> shift) & 255u;
-        const uint32_t peers = __match_any_sync(0xFFFFFFFFu, d);
-        const uint32_t rank = (uint32_t)__popc(peers & ((1u << lane) - 1u));
-        uint32_t base = 0;
-        if (rank == 0) {   // first lane with this digit: column `warp` of the histogram is this warp's alone
-          base = hist[d * kRadixHistStride + warp];
-          hist[d * kRadixHistStride + warp] = base + (uint32_t)__popc(peers);
+  for (int i = 0; i < E; ++i) v[i] = a[base + i];
+  for (int size = 2; size <= kMergeThreads * E; size <<= 1) {
+    const bool asc = (base & size) == 0;   // for size > E every key of the thread lies in the same half
+    for (int stride = size >> 1; stride >= E; stride >>= 1) {
+      const bool keep_min = ((base & stride) == 0) == asc;
+      if (stride >= 32 * E) {
+        // the partner of key i of thread t is key i of thread t ^ (stride / E), same lane of another warp: exchanged
+        // through shared memory laid out [i][thread], which neither the stores nor the loads conflict on
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < E; ++i) a[i * kMergeThreads + threadIdx.x] = v[i];
+        __syncthreads();
+        const int partner = threadIdx.x ^ (stride / E);
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+          const uint32_t other = a[i * kMergeThreads + partner];
+          v[i] = keep_min ? min(v[i], other) : max(v[i], other);
         }
-        base = __shfl_sync(0xFFFFFFFFu, base, __ffs((int)peers) - 1);
-        offs[j >> 1] |= (base + rank) << (16 * (j & 1));
-        __syncwarp();
-      }
-    }
-    __syncthreads();
-    // exclusive prefix sum of the histogram in digit-major, warp-minor order
-    {
-      const int first = threadIdx.x * kPer;
-      uint32_t sum = 0;
+      } else {
+        const int lane_mask = stride / E;
 #pragma unroll
-      for (int i = 0; i < kPer; ++i) sum += first + i < entries ? hist[first + i] : 0u;
-      uint32_t incl = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += up;
-      }
-      if (lane == 31) wsum[warp] = incl;
-      __syncthreads();
-      uint32_t run = incl - sum;
-      for (int w = 0; w < warp; ++w) run += wsum[w];
-#pragma unroll
-      for (int i = 0; i < kPer; ++i) {
-        if (first + i < entries) {
-          const uint32_t v = hist[first + i];
-          hist[first + i] = run;
-          run += v;
+        for (int i = 0; i < E; ++i) {
+          const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, v[i], lane_mask);
+          v[i] = keep_min ? min(v[i], other) : max(v[i], other);
         }
       }
     }
-    __syncthreads();
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      if (j < E) {
-        const uint32_t key = mine[32 * j];
-        const uint32_t d = (key >> shift) & 255u;
-        dst[hist[d * kRadixHistStride + warp] + ((offs[j >> 1] >> (16 * (j & 1))) & 0xFFFFu)] = key;
+    for (int sb = kLogE - 1; sb >= 0; --sb) {
+      const int st = 1 << sb;
+      if (st < size) {
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+          if ((i & st) == 0) {
+            const bool up = ((base + i) & size) == 0;   // within a thread the direction can differ while size <= E
+            const uint32_t lo = min(v[i], v[i | st]), hi = max(v[i], v[i | st]);
+            v[i] = up ? lo : hi;
+            v[i | st] = up ? hi : lo;
+          }
+        }
       }
     }
-    __syncthreads();
-    uint32_t* t = src; src = dst; dst = t;
   }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < E; ++i) a[base + i] = v[i];
+  __syncthreads();
 }
 
 // Launch shape of the merge for n old entries on `sms` SMs: entries per tile and number of tiles (>= 1).
@@ -896,7 +878,6 @@ merge_kernel(const float* __restrict__ old_buf, int n, const float* __restrict__
   uint32_t* const own_sorted = msm + k2; // [k2] the same, ascending
   uint32_t* const tkeys = msm + 2 * k2;  // [tile_len] keys of the tile's old entries
   __shared__ int own_count, below_count;
-  __shared__ uint32_t radix_hist[256 * kRadixHistStride], radix_wsum[kMergeThreads / 32];
   pdl_launch_dependents();
   pdl_wait();   // the new scores, the buffer and the index may come from the kernel before this one
   IndexSlot dst{};
@@ -923,16 +904,52 @@ merge_kernel(const float* __restrict__ old_buf, int n, const float* __restrict__
   for (int t = blockIdx.x; t < tiles; t += gridDim.x) {
     const int e0 = t * tile_len, e1 = min(n, e0 + tile_len), len = e1 - e0;
     const bool first = e0 == 0, last = t == tiles - 1;
-    const uint32_t lo = first ? 0u : key_of_bits(canonical_bits(old_buf[e0 - 1]));
-    const uint32_t hi = last ? 0u : key_of_bits(canonical_bits(old_buf[e1 - 1]));
+    // every global load of the round is issued before anything waits on one: the tile's range, its entries
+    // (at most 8 per thread) and the first 4096 new scores
+    const float lo_f = first ? 0.f : old_buf[e0 - 1];
+    const float hi_f = last ? 0.f : old_buf[e1 - 1];
+    float tv[kMergeTileMax / kMergeThreads], nv[4];
+#pragma unroll
+    for (int u = 0; u < kMergeTileMax / kMergeThreads; ++u) {
+      const int i = threadIdx.x + u * kMergeThreads;
+      tv[u] = i < len ? old_buf[e0 + i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = threadIdx.x + u * kMergeThreads;
+      nv[u] = j < k ? __ldg(new_scores + j) : 0.f;
+    }
+    const uint32_t lo = key_of_bits(canonical_bits(lo_f)), hi = key_of_bits(canonical_bits(hi_f));
     if (threadIdx.x == 0) { own_count = 0; below_count = 0; }
     __syncthreads();
-    for (int i = threadIdx.x; i < len; i += kMergeThreads) tkeys[i] = key_of_bits(canonical_bits(old_buf[e0 + i]));
+#pragma unroll
+    for (int u = 0; u < kMergeTileMax / kMergeThreads; ++u) {
+      const int i = threadIdx.x + u * kMergeThreads;
+      if (i < len) tkeys[i] = key_of_bits(canonical_bits(tv[u]));
+    }
     int below = 0;
-    for (int j = threadIdx.x; j < k; j += kMergeThreads) {
-      const uint32_t x = key_of_bits(canonical_bits(__ldg(new_scores + j)));
-      if (!first && x < lo) ++below;
-      else if (last || x < hi) own[atomicAdd(&own_count, 1)] = x;
+    for (int j0 = 0; j0 < k; j0 += kMergeThreads) {   // uniform trip count: the warp votes below
+      const int j = j0 + threadIdx.x;
+      float xf = 0.f;
+      if (j0 < 4 * kMergeThreads) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) xf = (j0 == u * kMergeThreads) ? nv[u] : xf;
+      } else if (j < k) {
+        xf = __ldg(new_scores + j);
+      }
+      const uint32_t x = key_of_bits(canonical_bits(xf));
+      const bool is_below = j < k && !first && x < lo;
+      const bool is_own = j < k && !is_below && (last || x < hi);
+      below += is_below ? 1 : 0;
+      // one shared-memory atomic per warp, not per key: a skewed batch sends every key to the same counter
+      const uint32_t votes = __ballot_sync(0xFFFFFFFFu, is_own);
+      if (votes) {
+        const int lane = threadIdx.x & 31, leader = __ffs((int)votes) - 1;
+        int base = 0;
+        if (lane == leader) base = atomicAdd(&own_count, __popc(votes));
+        base = __shfl_sync(0xFFFFFFFFu, base, leader);
+        if (is_own) own[base + __popc(votes & ((1u << lane) - 1u))] = x;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xFFFFFFFFu, below, o);
@@ -953,10 +970,18 @@ merge_kernel(const float* __restrict__ old_buf, int n, const float* __restrict__
       }
       __syncthreads();
     } else {
-      __syncthreads();   // every thread has read own_count
-      block_radix_sort(own, own_sorted, m, radix_hist, radix_wsum);
-      for (int i = threadIdx.x; i < m; i += kMergeThreads) own_sorted[i] = own[i];
+      // a skewed batch: this block owns hundreds or thousands of the new keys
+      int m2 = kMergeThreads;
+      while (m2 < m) m2 <<= 1;
+      for (int i = threadIdx.x; i < m2; i += kMergeThreads) own_sorted[i] = i < m ? own[i] : 0xFFFFFFFFu;
       __syncthreads();
+      switch (m2 / kMergeThreads) {
+        case 1: block_bitonic_sort<1>(own_sorted); break;
+        case 2: block_bitonic_sort<2>(own_sorted); break;
+        case 4: block_bitonic_sort<4>(own_sorted); break;
+        case 8: block_bitonic_sort<8>(own_sorted); break;
+        default: block_bitonic_sort<16>(own_sorted); break;
+      }
     }
     // ---- place the own keys: e0 + #{tile entries <= x} + c_below + i ----
     for (int i = threadIdx.x; i < m; i += kMergeThreads) {
@@ -1047,17 +1072,18 @@ classify_threshold_kernel(const float* __restrict__ scores, int64_t Nc, const fl
 
 // ---------------------------------------------------------------------------------------------
 // Budget report: the positions of the samples in stage 3 (the target takes over), in input order, and their
-// number B.  A stream compaction in one pass over the stage bytes: a block takes tiles of kIdsTile bytes in the
-// order of a ticket counter, counts the stage-3 bytes of its tile, publishes that count, obtains the number of
-// stage-3 bytes in all earlier tiles by looking back over the published words of its predecessors (each word
-// holds a tile's own count or, once known, the count of everything up to and including it), and writes its
-// positions.  Tickets are drawn in launch order, so the block that owns an earlier tile is always running or
+// number B.  A stream compaction in one pass over the stage bytes.  The bytes are cut into ranges of 4096 Q bytes
+// (Q <= 32 sixteen-byte pieces per thread); a block takes ranges in the order of a ticket counter.  For a range it
+// loads every byte once (all loads in flight together), keeps one bit per byte in registers, publishes the range's
+// count, sums the counts of all earlier ranges by looking back over their published words (a word holds a range's
+// own count or, once known, the count of everything up to and including it), and writes the positions from the
+// bits it kept.  Tickets are drawn in launch order, so the block that owns an earlier range is always running or
 // done: the look-back cannot wait on a block that has not started.  Every wait is bounded all the same.
 // Everything is integer work in a fixed order: the result is unique.
 // ---------------------------------------------------------------------------------------------
 constexpr int kIdsThreads = 256;
-constexpr int kIdsPerThread = 32;                       // two 16-byte pieces per thread
-constexpr int kIdsTile = kIdsThreads * kIdsPerThread;   // 8192 stage bytes per tile
+constexpr int kIdsMaxRows = 32;                          // 16-byte pieces per thread at most
+constexpr int kIdsRowBytes = kIdsThreads * 16;           // 4096 stage bytes per row of pieces
 constexpr unsigned long long kIdsOwnCount = 1ull << 32, kIdsPrefixKnown = 2ull << 32;
 constexpr int kIdsSpinLimit = 1 << 22;
 
@@ -1069,7 +1095,13 @@ __device__ __forceinline__ uint32_t stage3_mask16(const uint8_t* __restrict__ st
     const uint4 q = *reinterpret_cast<const uint4*>(stage + j);
     const uint32_t w[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-    for (int i = 0; i < 16; ++i) m16 |= (((w[i >> 2] >> (8 * (i & 3))) & 0xFFu) == 3u ? 1u : 0u) << i;
+    for (int i = 0; i < 4; ++i) {
+      // a byte equals 3 iff (byte ^ 3) is zero: the classic zero-byte test, exact, on four bytes at once; the
+      // multiplication then gathers bit 0 of the four bytes into bits 24 .. 27 (no two partial products meet)
+      const uint32_t x = w[i] ^ 0x03030303u;
+      const uint32_t z = ~(((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x | 0x7F7F7F7Fu);   // 0x80 in every byte that was 3
+      m16 |= ((((z >> 7) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
+    }
   } else {
     for (int i = 0; i < 16 && j + i < Nc; ++i) m16 |= (stage[j + i] == 3 ? 1u : 0u) << i;
   }
@@ -1082,39 +1114,37 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
   return v;
 }
 
-// state: one word per tile (zero before the launch), ticket: one counter (zero before the launch); both unused
-// (may be nullptr) when there is a single tile.
+// state: one word per range (zero before the launch), ticket: one counter (zero before the launch); both unused
+// (may be nullptr) when there is a single range.
 __global__ void __launch_bounds__(kIdsThreads)
-takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int tiles, bool vec,
+takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int Q, int ranges, bool vec,
                     unsigned long long* __restrict__ state, unsigned int* __restrict__ ticket,
                     int32_t* __restrict__ ids, int64_t ids_cap, uint32_t* __restrict__ count,
                     unsigned int* __restrict__ dev_status) {
-  __shared__ int32_t staged[kIdsTile];
   __shared__ uint32_t warp_total[kIdsThreads / 32];
-  __shared__ uint32_t tile_sh, prefix_sh;
+  __shared__ uint32_t range_sh, prefix_sh;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (;;) {
-    if (threadIdx.x == 0) tile_sh = tiles == 1 ? blockIdx.x : atomicAdd(ticket, 1u);
+    if (threadIdx.x == 0) range_sh = ranges == 1 ? 0u : atomicAdd(ticket, 1u);
     __syncthreads();
-    const int tile = (int)tile_sh;
-    if (tile >= tiles) return;
-    // A warp covers 1024 consecutive bytes as two rows of 512: lane l holds bytes [16 l, 16 l + 16) of each row, so
+    const int range = (int)range_sh;
+    if (range >= ranges) return;
+    // A warp covers 512 Q consecutive bytes as Q rows of 512: lane l holds bytes [16 l, 16 l + 16) of each row, so
     // every load instruction of the warp reads 512 contiguous bytes.
-    const int64_t warp_base = (int64_t)tile * kIdsTile + (int64_t)warp * (kIdsPerThread * 32);
-    uint32_t m[2], excl[2], row_total[2];
+    const int64_t warp_base = (int64_t)range * Q * kIdsRowBytes + (int64_t)warp * Q * 512;
+    uint32_t m[kIdsMaxRows / 2];   // two 16-bit masks per word
+    uint32_t mine = 0;
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      m[r] = stage3_mask16(stage, warp_base + r * 512 + lane * 16, Nc, vec);
-      uint32_t incl = (uint32_t)__popc(m[r]);
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += up;
-      }
-      excl[r] = incl - (uint32_t)__popc(m[r]);
-      row_total[r] = __shfl_sync(0xFFFFFFFFu, incl, 31);
+    for (int q = 0; q < kIdsMaxRows; q += 2) {
+      const uint32_t a = q < Q ? stage3_mask16(stage, warp_base + q * 512 + lane * 16, Nc, vec) : 0u;
+      const uint32_t b = q + 1 < Q ? stage3_mask16(stage, warp_base + (q + 1) * 512 + lane * 16, Nc, vec) : 0u;
+      m[q >> 1] = a | (b << 16);
+      mine += (uint32_t)__popc(m[q >> 1]);
     }
-    if (lane == 0) warp_total[warp] = row_total[0] + row_total[1];
+    uint32_t wsum = mine;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
+    if (lane == 0) warp_total[warp] = wsum;
     __syncthreads();
     uint32_t warp_off = 0, total = 0;
 #pragma unroll
@@ -1123,27 +1153,23 @@ takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int tiles, bo
       warp_off += w < warp ? t : 0u;
       total += t;
     }
-    // positions of this tile, in order, into shared memory
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      uint32_t loc = warp_off + (r ? row_total[0] : 0u) + excl[r];
-      const int32_t first = (int32_t)(warp_base + r * 512 + lane * 16);
-      for (uint32_t mm = m[r]; mm != 0u; mm &= mm - 1u) staged[loc++] = first + (__ffs((int)mm) - 1);
-    }
-    // number of stage-3 bytes in all earlier tiles
+    // number of stage-3 bytes in all earlier ranges
     if (warp == 0) {
       uint32_t prefix = 0;
-      if (tiles > 1) {
-        if (lane == 0) {
-          __threadfence();
-          atomicExch(state + tile, (tile == 0 ? kIdsPrefixKnown : kIdsOwnCount) | total);
-        }
+      if (ranges > 1) {
+        if (lane == 0) atomicExch(state + range, (range == 0 ? kIdsPrefixKnown : kIdsOwnCount) | total);
         int spins = 0;
-        for (int p0 = tile - 1; p0 >= 0; ) {
-          const int p = p0 - lane;
-          const unsigned long long w = p >= 0 ? ld_relaxed_u64(state + p) : kIdsPrefixKnown;
-          const uint32_t ready = __ballot_sync(0xFFFFFFFFu, (w >> 32) != 0ull);
-          if (ready != 0xFFFFFFFFu) {
+        bool found = false;
+        for (int p0 = range - 1; p0 >= 0 && !found; ) {
+          // four windows of 32 predecessors, nearest first; their loads are independent
+          unsigned long long w[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int p = p0 - 32 * u - lane;
+            w[u] = p >= 0 ? ld_relaxed_u64(state + p) : kIdsPrefixKnown;
+          }
+          const bool mine_ready = (w[0] >> 32) != 0ull && (w[1] >> 32) != 0ull && (w[2] >> 32) != 0ull && (w[3] >> 32) != 0ull;
+          if (!__all_sync(0xFFFFFFFFu, mine_ready)) {
             if (++spins > kIdsSpinLimit) {   // cannot happen with tickets in launch order; give up rather than hang
               if (lane == 0) atomicOr(dev_status, 2u);
               break;
@@ -1151,28 +1177,54 @@ takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int tiles, bo
             __nanosleep(20);
             continue;
           }
-          const uint32_t known = __ballot_sync(0xFFFFFFFFu, (w >> 32) == 2ull);
-          const int stop = known ? __ffs((int)known) - 1 : 31;   // nearest predecessor whose prefix is known
-          uint32_t v = lane <= stop ? (uint32_t)w : 0u;
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-          prefix += v;
-          if (known) break;
-          p0 -= 32;
+          for (int u = 0; u < 4; ++u) {
+            if (found) continue;
+            const uint32_t known = __ballot_sync(0xFFFFFFFFu, (w[u] >> 32) == 2ull);
+            const int stop = known ? __ffs((int)known) - 1 : 31;   // nearest predecessor whose prefix is known
+            uint32_t v = lane <= stop ? (uint32_t)w[u] : 0u;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+            prefix += v;
+            found = known != 0u;
+          }
+          p0 -= 128;
         }
-        if (lane == 0 && tile > 0) atomicExch(state + tile, kIdsPrefixKnown | (unsigned long long)(prefix + total));
+        if (lane == 0 && range > 0) atomicExch(state + range, kIdsPrefixKnown | (unsigned long long)(prefix + total));
       }
       if (lane == 0) {
         prefix_sh = prefix;
-        if (tile == tiles - 1 && count != nullptr) *count = prefix + total;
+        if (range == ranges - 1 && count != nullptr) *count = prefix + total;
       }
     }
     __syncthreads();
-    const int64_t prefix = prefix_sh;
-    for (uint32_t t = threadIdx.x; t < total; t += kIdsThreads)
-      if (prefix + t < ids_cap) ids[prefix + t] = staged[t];
-    if (tiles == 1) return;
-    __syncthreads();   // the shared words are reused by the next tile
+    // positions, row by row: a row's positions are consecutive in the output
+    int64_t row_pos = (int64_t)prefix_sh + warp_off;
+#pragma unroll
+    for (int q = 0; q < kIdsMaxRows; ++q) {
+      if (q < Q) {
+        const uint32_t mm = (m[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
+        uint32_t incl = (uint32_t)__popc(mm);
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += up;
+        }
+        const int64_t pos = row_pos + incl - (uint32_t)__popc(mm);
+        const int32_t first = (int32_t)(warp_base + q * 512 + lane * 16) - 1;
+        int32_t* dst_id = ids + pos;
+        if (pos + 16 <= ids_cap) {   // the usual case: no bounds test per position
+          for (uint32_t r = mm; r != 0u; r &= r - 1u) *dst_id++ = first + __ffs((int)r);
+        } else {
+          int64_t at = pos;
+          for (uint32_t r = mm; r != 0u; r &= r - 1u, ++at)
+            if (at < ids_cap) ids[at] = first + __ffs((int)r);
+        }
+        row_pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      }
+    }
+    if (ranges == 1) return;
+    __syncthreads();   // every thread is done with the shared words of this round
   }
 }
 

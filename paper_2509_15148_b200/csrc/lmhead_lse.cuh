@@ -18,7 +18,7 @@ constexpr int kBlockK = 64;    // bf16 elements per shared-memory stage row (128
 constexpr int kUmmaK = 16;     // K of one tcgen05.mma (kind::f16)
 constexpr int kScoreThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer, warps 2-5: epilogue
 constexpr int kTmemCols = 512;      // two 256-column accumulators
-constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s: far beyond any legitimate wait
+constexpr long long kWaitLimitCycles = 4000000000LL;  // default bound of a pipeline wait, ~2 s: far beyond any legitimate one
 
 // Two forms of the kernel.  CTAS = 1: every CTA computes 128 x 256 tiles on its own.  CTAS = 2: the two CTAs
 // of a cluster compute one 256 x 256 tile with tcgen05.mma.cta_group::2; each loads its own 128 rows of H and
@@ -53,6 +53,8 @@ struct ScorePlan {
   int M_pad;   // RB * rows per unit
   int ctas;    // 1 or 2: CTAs per worker
   int vocab_offset;  // id of this W's first row (0 unless W is a slice of a sharded vocabulary)
+  long long wait_limit;  // cycles after which a pipeline wait gives up (the host's setting; kWaitLimitCycles by default)
+  int withhold_loads;    // diagnostic: the producer issues no loads, so the first wait for data must run out
 };
 
 __host__ __device__ inline void decode_unit(const ScorePlan& p, int u, int& rb, int& c, int& nt0, int& nt1) {
@@ -125,18 +127,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up when another thread of the CTA has raised `abort` or after
-// kWaitLimitCycles, in which case it raises `abort` itself.  Returns false when it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort) {
+// Bounded wait: gives up when another thread of the CTA has raised `abort` or after `limit` cycles, in which
+// case it raises `abort` itself - and, in a CTA pair, the flag of the other CTA too (`peer_abort`, an address in
+// the cluster's shared window, 0 for a single CTA), so that both leave together.  Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort, long long limit,
+                                          uint32_t peer_abort) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   uint32_t spins = 0;
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 0xFFu) == 0u) {
+    if ((++spins & 7u) == 0u) {
       if (*abort) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit) {
         *abort = 1u;
+        if (peer_abort) asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_abort), "r"(1u) : "memory");
         return false;
       }
     }
@@ -275,6 +280,8 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;   // 0 = leader
+  const long long wait_limit = plan.wait_limit;
+  const uint32_t peer_abort = CTAS == 2 ? map_to_cta(smem_u32((const void*)abort_flag), rank ^ 1u) : 0u;
   const int worker = blockIdx.x / CTAS;
   const int workers = gridDim.x / CTAS;
 
@@ -309,7 +316,7 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
 
   if (warp == 0) {
     // ---------------- TMA producer (every CTA loads its own operand halves) ----------------
-    if (lane == 0) {
+    if (lane == 0 && !plan.withhold_loads) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -320,7 +327,7 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
         for (int nt = nt0; nt < nt1 && ok; ++nt) {
           const int col0 = nt * kBlockN + (int)rank * Cfg::kBRows;
           for (int kb = 0; kb < plan.KB; ++kb) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, wait_limit, peer_abort)) { ok = false; break; }
             const uint32_t sa = smem_base + (uint32_t)stage * Cfg::kStageBytes;
             if (CTAS == 1) {
               mbar_expect_tx(full_bar(stage), Cfg::kStageBytes);
@@ -350,11 +357,11 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
         int rb, c, nt0, nt1;
         decode_unit(plan, u, rb, c, nt0, nt1);
         for (int nt = nt0; nt < nt1 && ok; ++nt) {
-          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, wait_limit, peer_abort)) { ok = false; break; }
           tc_fence_after();
           const uint32_t tmem_d = tmem_base + (uint32_t)acc * kBlockN;
           for (int kb = 0; kb < plan.KB; ++kb) {
-            if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(full_bar(stage), phase, abort_flag, wait_limit, peer_abort)) { ok = false; break; }
             tc_fence_after();
             const uint32_t sa = smem_base + (uint32_t)stage * Cfg::kStageBytes;
             const uint64_t da = umma_smem_desc(sa);
@@ -399,7 +406,7 @@ lmhead_lse_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_const
       const float kScale = rs * kLog2e;
       float m = -INFINITY, l = 0.f;
       for (int nt = nt0; nt < nt1; ++nt) {
-        if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, wait_limit, peer_abort)) { ok = false; break; }
         tc_fence_after();
         const int n0 = nt * kBlockN;
         const uint32_t taddr = tmem_base + lane_base + (uint32_t)(acc * kBlockN);

@@ -176,3 +176,43 @@ def test_conformal_stress_whole_sequence_with_index_in_one_graph():
         assert np.array_equal(host_u32(counts[a]), want_counts)
     assert np.array_equal(f32_bits(buf), f32_bits(orc.calib_update(calib, news_h[-1])))
     assert binding.last_device_status() == 0
+
+
+def test_conformal_stress_every_step_eager_with_index():
+    """All 64 steps of the conformal-only workload through the indexed calls, launched one by one, with the
+    numerators, p-value bits, the three rows of stage bytes, their counts and the buffer checked against the
+    oracle after every step (the oracle replays the same inserts)."""
+    cfg = inputs.CONFORMAL_STRESS
+    Nc, n0, k, steps, alphas = cfg["Nc"], cfg["n0"], cfg["k"], cfg["steps"], cfg["alphas"]
+    scores = inputs.lognormal_scores(inputs.BASE_SEED + 1, Nc)
+    calib = np.sort(inputs.lognormal_scores(inputs.BASE_SEED + 2, n0))
+    cap = n0 + k * steps
+    s_dev = dev(scores)
+    buf = poison((cap,), torch.float32)
+    buf[:n0] = dev(calib)
+    numer, p = poison((Nc,), torch.int32), poison((Nc,), torch.float32)
+    stage, counts = poison((len(alphas), Nc), torch.uint8), poison((len(alphas), 3), torch.int32)
+    index = workspace(binding.calib_index_bytes(cap))
+    ws = workspace(binding.calib_workspace_bytes(cap, k))
+    binding.calib_index_build(buf, n0, index)
+    n = n0
+    for t in range(steps):
+        new = inputs.lognormal_scores(inputs.BASE_SEED + 3 + t, k)
+        for out in (numer, p, stage, counts):
+            out.view(torch.uint8).fill_(0xFF)
+        binding.rank_classify_indexed(s_dev, buf, n, index, alphas, numer, p, stage, counts)
+        n_next = binding.calib_update_indexed(buf, n, dev(new), index, ws)
+        torch.cuda.synchronize()
+        want_numer = orc.conformal_numer_sorted(scores, calib)
+        assert np.array_equal(host_u32(numer), want_numer), t
+        assert np.array_equal(f32_bits(p), f32_bits(orc.pvalue(want_numer, n))), t
+        for a, alpha in enumerate(alphas):
+            want_stage, want_counts = orc.classify(want_numer, n, alpha)
+            assert np.array_equal(stage[a].cpu().numpy(), want_stage), (t, alpha)
+            assert np.array_equal(host_u32(counts[a]), want_counts), (t, alpha)
+        calib = orc.calib_update(calib, new)
+        assert n_next == calib.size
+        assert np.array_equal(f32_bits(buf[:n_next]), f32_bits(calib)), t
+        n = n_next
+    assert n == cap and np.all(np.diff(calib) >= 0)
+    assert binding.last_device_status() == 0
