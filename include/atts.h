@@ -199,7 +199,10 @@ int atts_rank_classify(const float* scores, int64_t Nc, const float* calib_sorte
  * Sampling", Sec. 3.3: the target model continues exactly those): the positions of the samples whose stage is
  * ATTS_STAGE_TARGET, ascending, and their number B.
  *
- *   stage         dev  [Nc] uint8, as written by atts_classify (a row of atts_rank_classify's output)
+ *   stage         dev  [Nc] uint8, as written by atts_classify (a row of atts_rank_classify's output); only the value
+ *                      ATTS_STAGE_TARGET counts, any other byte value is skipped.  Any alignment: the kernel reads the
+ *                      aligned 16-byte pieces that hold the array, so up to 15 bytes before stage[0], inside the
+ *                      piece that holds it, are read and ignored
  *   ids           dev  [ids_cap] int32 out: the first min(B, ids_cap) positions; may be NULL when ids_cap == 0
  *   count         dev  [1] uint32 out: B (also when B > ids_cap); may be NULL
  *   workspace     dev  256-byte aligned, at least atts_takeover_ids_workspace_bytes(Nc) bytes

@@ -114,6 +114,7 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaFuncSetAttribute(small_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       4 * (kSmallUpdMaxOld + kSmallUpdMaxNew)) == cudaSuccess;
       const int merge_smem = 4 * (2 * kSortMaxK + kMergeTileMax);
+      ok = ok && cudaFuncSetAttribute(takeover_ids_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kIdsSmemBytes) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(merge_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, merge_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(merge_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, merge_smem) == cudaSuccess;
       if (!ok) {
@@ -574,11 +575,11 @@ int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, u
 }
 
 // Workspace of atts_takeover_ids: [one 64-bit word per range][ticket counter], cleared before the launch.  A range
-// is at least 4096 stage bytes, which bounds the number of ranges whatever the device.
+// is at least 8192 stage bytes, which bounds the number of ranges whatever the device.
 int atts_takeover_ids_workspace_bytes(int64_t Nc, size_t* bytes) {
   if (!bytes) return ATTS_ERR_NULL;
   if (Nc < 0 || Nc >= (1ll << 31)) return ATTS_ERR_SHAPE;
-  *bytes = round_up((size_t)((Nc + kIdsRowBytes - 1) / kIdsRowBytes) * sizeof(unsigned long long) + 8, 256) + 256;
+  *bytes = round_up((size_t)((Nc + 16 + kIdsRowBytes - 1) / kIdsRowBytes) * sizeof(unsigned long long) + 8, 256) + 256;
   return ATTS_OK;
 }
 
@@ -601,21 +602,26 @@ int atts_takeover_ids(const uint8_t* stage, int64_t Nc, int32_t* ids, int64_t id
     }
     return ATTS_OK;
   }
-  // about four ranges per SM, a range being Q rows of 4096 bytes (1 <= Q <= 32)
-  const int64_t per_range = (Nc + (int64_t)di->sm_count * 4 - 1) / ((int64_t)di->sm_count * 4);
-  int64_t Q = (per_range + kIdsRowBytes - 1) / kIdsRowBytes;
-  Q = Q < 1 ? 1 : (Q > kIdsMaxRows ? kIdsMaxRows : Q);
-  const int ranges = (int)((Nc + Q * kIdsRowBytes - 1) / (Q * kIdsRowBytes));
-  const bool vec = aligned(stage, 16);
+  // A range is Q rows of 4096 bytes, Q even, 2 <= Q <= 8.  Long ranges even out the lanes' work and cost less per
+  // byte, so Q grows as soon as every block that fits the GPU (four per SM) has a range.  The kernel reads whole
+  // 16-byte pieces: it starts at the boundary at or below the first stage byte and is told how many bytes to skip.
+  const int head = (int)(reinterpret_cast<uintptr_t>(stage) & 15u);
+  const uint8_t* base = stage - head;
+  const int64_t len = Nc + head;
+  const int64_t slots = (int64_t)di->sm_count * 4;
+  int64_t Q = (len + kIdsRowBytes * slots - 1) / (kIdsRowBytes * slots);
+  Q = (Q + 1) & ~1ll;
+  Q = Q < 2 ? 2 : (Q > kIdsMaxRows ? kIdsMaxRows : Q);
+  const int ranges = (int)((len + Q * kIdsRowBytes - 1) / (Q * kIdsRowBytes));
   unsigned long long* state = static_cast<unsigned long long*>(workspace);
   unsigned int* ticket = reinterpret_cast<unsigned int*>(state + ranges);
   if (ranges > 1 && cudaMemsetAsync(workspace, 0, (size_t)ranges * sizeof(unsigned long long) + 8, stream) != cudaSuccess) {
     cudaGetLastError();
     return ATTS_ERR_CUDA;
   }
-  const int blocks = ranges < di->sm_count * 8 ? ranges : di->sm_count * 8;
-  takeover_ids_kernel<<<blocks, kIdsThreads, 0, stream>>>(stage, Nc, (int)Q, ranges, vec, state, ticket, ids, ids_cap, count,
-                                                         di->dev_status);
+  const int blocks = ranges < slots ? ranges : (int)slots;
+  takeover_ids_kernel<<<blocks, kIdsThreads, kIdsSmemBytes, stream>>>(base, len, head, (int)Q, ranges, state, ticket, ids, ids_cap,
+                                                                     count, di->dev_status);
   return launch_status();
 }
 

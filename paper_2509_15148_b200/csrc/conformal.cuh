@@ -1072,40 +1072,62 @@ classify_threshold_kernel(const float* __restrict__ scores, int64_t Nc, const fl
 
 // ---------------------------------------------------------------------------------------------
 // Budget report: the positions of the samples in stage 3 (the target takes over), in input order, and their
-// number B.  A stream compaction in one pass over the stage bytes.  The bytes are cut into ranges of 4096 Q bytes
-// (Q <= 32 sixteen-byte pieces per thread); a block takes ranges in the order of a ticket counter.  For a range it
-// loads every byte once (all loads in flight together), keeps one bit per byte in registers, publishes the range's
-// count, sums the counts of all earlier ranges by looking back over their published words (a word holds a range's
-// own count or, once known, the count of everything up to and including it), and writes the positions from the
-// bits it kept.  Tickets are drawn in launch order, so the block that owns an earlier range is always running or
-// done: the look-back cannot wait on a block that has not started.  Every wait is bounded all the same.
-// Everything is integer work in a fixed order: the result is unique.
+// number B.  A stream compaction in one pass over the stage bytes.  Its arithmetic is light, so what decides the
+// time is how few instructions a byte costs and whether the loads of the next piece of work are in flight while
+// the present one is being expanded.
+//
+// The bytes, counted from the 16-byte boundary at or below the first one (`head` bytes earlier, never counted), are
+// cut into ranges of 4096 Q bytes (Q even, <= 8: at most 32,768 bytes, so a position inside a range fits in 16
+// bits); a block takes ranges in the order of a ticket counter, one ticket ahead of the range it works on.  For a range,
+//  1. every thread has copied Q pieces of 16 bytes into shared memory with asynchronous copies issued while the
+//     range before was being worked on (a warp's copy instruction covers 512 contiguous bytes; bytes past the end
+//     arrive as zeros); it reads its own pieces back, turns each into 16 bits (bit set where the byte is 3) and
+//     stores them in shared memory, where they form a bit map of the warp's 512 Q bytes in input order; then it
+//     issues the copies of the next range into the slots it has just read;
+//  2. every lane then owns 16 Q consecutive bits of that map, i.e. a contiguous piece of the input, so that one
+//     prefix sum per warp (not one per row) gives the place of its first position, and its positions are consecutive;
+//  3. the block publishes the range's count and sums the counts of all earlier ranges by looking back over their
+//     published words (a word holds a range's own count or, once known, the count of everything up to and including
+//     it) while the other warps already expand their bits into 16-bit positions in shared memory;
+//  4. the staged positions are written out by the whole block, 32 consecutive words per warp instruction (a lane
+//     writing its own short run straight to global memory would send eight partial sectors where one whole one does).
+// A range with more stage-3 bytes than the staging area holds (more than a quarter of a full range) is written
+// directly from the bit map, slower but the same result.
+// Tickets are drawn in launch order and a block works through its tickets in increasing order, so the block that
+// owns an earlier range is always running or done: the look-back cannot wait on a block that has not started.
+// Every wait is bounded all the same.  Everything is integer work in a fixed order: the result is unique.
 // ---------------------------------------------------------------------------------------------
 constexpr int kIdsThreads = 256;
-constexpr int kIdsMaxRows = 32;                          // 16-byte pieces per thread at most
+constexpr int kIdsMaxRows = 8;                           // 16-byte pieces per thread at most
 constexpr int kIdsRowBytes = kIdsThreads * 16;           // 4096 stage bytes per row of pieces
+constexpr int kIdsStageCap = 7680;                       // positions staged per range (four blocks fit an SM)
+constexpr int kIdsSmemBytes = kIdsMaxRows * kIdsRowBytes + 2 * (kIdsThreads / 32) * kIdsMaxRows * 64 + 2 * kIdsStageCap;
 constexpr unsigned long long kIdsOwnCount = 1ull << 32, kIdsPrefixKnown = 2ull << 32;
 constexpr int kIdsSpinLimit = 1 << 22;
 
-// Bit i of the result is set where byte i of the 16 stage bytes at stage + j is 3 (bytes beyond Nc are not).
-__device__ __forceinline__ uint32_t stage3_mask16(const uint8_t* __restrict__ stage, int64_t j, int64_t Nc, bool vec) {
-  uint32_t m16 = 0;
-  if (j >= Nc) return 0u;
-  if (vec && j + 16 <= Nc) {
-    const uint4 q = *reinterpret_cast<const uint4*>(stage + j);
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+// Bit i of the result is set where byte i of the 16 bytes is 3.
+__device__ __forceinline__ uint32_t stage3_mask16(const uint4& q) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  uint32_t acc = 0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      // a byte equals 3 iff (byte ^ 3) is zero: the classic zero-byte test, exact, on four bytes at once; the
-      // multiplication then gathers bit 0 of the four bytes into bits 24 .. 27 (no two partial products meet)
-      const uint32_t x = w[i] ^ 0x03030303u;
-      const uint32_t z = ~(((x & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | x | 0x7F7F7F7Fu);   // 0x80 in every byte that was 3
-      m16 |= ((((z >> 7) & 0x01010101u) * 0x01020408u) >> 24) << (4 * i);
-    }
-  } else {
-    for (int i = 0; i < 16 && j + i < Nc; ++i) m16 |= (stage[j + i] == 3 ? 1u : 0u) << i;
+  for (int i = 3; i >= 0; --i) {
+    // A byte equals 3 iff (byte ^ 3) is zero: the zero-byte test on four bytes at once, exact (bit 7 of a byte of
+    // t is set iff its low seven bits are not all zero; bit 7 of byte ^ 3 is bit 7 of the byte).  z has 0x80 in
+    // every byte that was 3.  The multiplication moves bits 7, 15, 23, 31 to bits 28 .. 31 (no two partial
+    // products meet, so nothing carries), and the funnel shift appends those four bits below the ones gathered
+    // so far: the last word handled, word 0, ends in bits 0 .. 3.
+    const uint32_t t = ((w[i] ^ 0x03030303u) & 0x7F7F7F7Fu) + 0x7F7F7F7Fu;
+    const uint32_t z = ~(t | w[i] | 0x7F7F7F7Fu);
+    acc = __funnelshift_l(z * 0x00204081u, acc, 4);
   }
-  return m16;
+  return acc;
+}
+
+// x >> n for n up to 32 (the hardware's shift gives zero for n = 32, which the language leaves undefined)
+__device__ __forceinline__ uint32_t shr_clamped(uint32_t x, uint32_t n) {
+  uint32_t y;
+  asm("shr.b32 %0, %1, %2;" : "=r"(y) : "r"(x), "r"(n));
+  return y;
 }
 
 __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
@@ -1114,62 +1136,168 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
   return v;
 }
 
+// The Q asynchronous 16-byte copies of one thread for the range that starts `range_base` bytes after `base`
+// (16-byte aligned); `len` bytes from `base` on exist, pieces beyond them arrive (partly) as zeros.
+__device__ __forceinline__ void ids_prefetch(const uint8_t* __restrict__ base, int64_t len, int64_t range_base, int Q,
+                                             uint4* raw) {
+  const int64_t j0 = range_base + (int64_t)(threadIdx.x >> 5) * Q * 512 + (threadIdx.x & 31) * 16;
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(raw + threadIdx.x);
+  if (range_base + (int64_t)Q * kIdsRowBytes <= len) {   // the whole range exists: nothing to test per piece
+    const uint8_t* src = base + j0;
+#pragma unroll
+    for (int q = 0; q < kIdsMaxRows; ++q)
+      if (q < Q)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + q * kIdsRowBytes), "l"(src + q * 512) : "memory");
+  } else {
+    for (int q = 0; q < Q; ++q) {
+      const int64_t j = j0 + q * 512;
+      const int64_t left = len - j;
+      const uint32_t valid = left >= 16 ? 16u : (left > 0 ? (uint32_t)left : 0u);
+      const uint8_t* src = base + (valid ? j : 0);
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + q * kIdsRowBytes), "l"(src), "r"(valid) : "memory");
+    }
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
 // state: one word per range (zero before the launch), ticket: one counter (zero before the launch); both unused
-// (may be nullptr) when there is a single range.
+// (may be nullptr) when there is a single range.  base: the 16-byte boundary at or below the first stage byte, which
+// is byte `head` from there; len = head + number of stage bytes.  Q: rows per range, even, 2 <= Q <= kIdsMaxRows.
+//
+// The loop is staggered by one turn: turn k reads range k and counts it, publishes that count, and then expands and
+// writes out range k - 1, whose look-back (the only step that depends on other blocks) has had a whole turn for its
+// predecessors' counts to appear; its loads are issued before the expansion and looked at after it.
 __global__ void __launch_bounds__(kIdsThreads)
-takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int Q, int ranges, bool vec,
+takeover_ids_kernel(const uint8_t* __restrict__ base, int64_t len, int head, int Q, int ranges,
                     unsigned long long* __restrict__ state, unsigned int* __restrict__ ticket,
                     int32_t* __restrict__ ids, int64_t ids_cap, uint32_t* __restrict__ count,
                     unsigned int* __restrict__ dev_status) {
-  __shared__ uint32_t warp_total[kIdsThreads / 32];
-  __shared__ uint32_t range_sh, prefix_sh;
+  extern __shared__ uint4 ids_smem[];
+  uint4* const raw = ids_smem;                                                                  // [Q][256] pieces
+  uint32_t* const bitmap = reinterpret_cast<uint32_t*>(ids_smem + kIdsMaxRows * kIdsThreads);   // [2][warps][128]: one bit per byte
+  uint16_t* const staged = reinterpret_cast<uint16_t*>(bitmap + 2 * (kIdsThreads / 32) * kIdsMaxRows * 16);
+  __shared__ uint32_t warp_total[2][kIdsThreads / 32];
+  __shared__ uint32_t range_sh[2], prefix_sh;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (;;) {
-    if (threadIdx.x == 0) range_sh = ranges == 1 ? 0u : atomicAdd(ticket, 1u);
-    __syncthreads();
-    const int range = (int)range_sh;
-    if (range >= ranges) return;
-    // A warp covers 512 Q consecutive bytes as Q rows of 512: lane l holds bytes [16 l, 16 l + 16) of each row, so
-    // every load instruction of the warp reads 512 contiguous bytes.
-    const int64_t warp_base = (int64_t)range * Q * kIdsRowBytes + (int64_t)warp * Q * 512;
-    uint32_t m[kIdsMaxRows / 2];   // two 16-bit masks per word
-    uint32_t mine = 0;
+  const int words = Q >> 1;   // bit-map words per lane
+  const int64_t range_bytes = (int64_t)Q * kIdsRowBytes;
+  const uint32_t warp_first = (uint32_t)(warp * Q * 512);   // of the warp's bytes, inside the range
+
+  // Thread 0 draws tickets two ranges ahead and keeps the newest in a register, so that the counter's round trip
+  // is over long before the value is needed.
+  uint32_t drawn = (uint32_t)ranges;
+  if (threadIdx.x == 0) {
+    range_sh[0] = ranges == 1 ? 0u : atomicAdd(ticket, 1u);
+    if (ranges > 1) drawn = atomicAdd(ticket, 1u);
+  }
+  __syncthreads();
+  int range = (int)range_sh[0];
+  if (range < ranges) ids_prefetch(base, len, range * range_bytes, Q, raw);
+  int prev = -1;                                  // the range counted in the turn before, to be written out in this one
+  uint32_t prev_local = 0, prev_mine = 0, prev_turns = 0, prev_total = 0;
+  for (int k = 0;; ++k) {
+    const bool cur = range < ranges;
+    if (!cur && prev < 0) break;
+    uint32_t* const wmap = bitmap + ((k & 1) * (kIdsThreads / 32) + warp) * (kIdsMaxRows * 16);
+    uint32_t mine = 0, incl = 0, turns = 0;
+    if (cur) {
+      // 1. lane l holds bytes [16 l, 16 l + 16) of each of the warp's Q rows of 512 bytes: its own copies have landed
+      uint16_t* const rows16 = reinterpret_cast<uint16_t*>(wmap);
+      asm volatile("cp.async.wait_all;" ::: "memory");
 #pragma unroll
-    for (int q = 0; q < kIdsMaxRows; q += 2) {
-      const uint32_t a = q < Q ? stage3_mask16(stage, warp_base + q * 512 + lane * 16, Nc, vec) : 0u;
-      const uint32_t b = q + 1 < Q ? stage3_mask16(stage, warp_base + (q + 1) * 512 + lane * 16, Nc, vec) : 0u;
-      m[q >> 1] = a | (b << 16);
-      mine += (uint32_t)__popc(m[q >> 1]);
+      for (int q = 0; q < kIdsMaxRows; ++q)
+        if (q < Q) rows16[q * 32 + lane] = (uint16_t)stage3_mask16(raw[q * kIdsThreads + threadIdx.x]);
+      if (range == 0 && threadIdx.x == 0) rows16[0] &= (uint16_t)(0xFFFFu << head);   // bytes before the first stage byte
+      __syncwarp();
+      // 2. lane l owns words [l Q/2, (l + 1) Q/2) of the warp's map = bytes [16 Q l, 16 Q (l + 1)) of the warp
+      const uint32_t* const seg = wmap + lane * words;
+      for (int i = 0; i < words; ++i) {
+        const uint32_t c = (uint32_t)__popc(seg[i]);
+        mine += c;
+        turns += max(c, 1u);   // iterations of the expansion loop: one per bit and one per empty word
+      }
+      incl = mine;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) turns = max(turns, __shfl_xor_sync(0xFFFFFFFFu, turns, o));
+      if (lane == 31) warp_total[k & 1][warp] = incl;
     }
-    uint32_t wsum = mine;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xFFFFFFFFu, wsum, o);
-    if (lane == 0) warp_total[warp] = wsum;
+    if (threadIdx.x == 0) {
+      range_sh[(k + 1) & 1] = drawn;   // the range after this one
+      drawn = (ranges > 1 && drawn < (uint32_t)ranges) ? atomicAdd(ticket, 1u) : (uint32_t)ranges;
+    }
     __syncthreads();
+    const int next = cur ? (int)range_sh[(k + 1) & 1] : ranges;
+    if (next < ranges) ids_prefetch(base, len, next * range_bytes, Q, raw);   // into the slots this thread has read
     uint32_t warp_off = 0, total = 0;
+    if (cur) {
 #pragma unroll
-    for (int w = 0; w < kIdsThreads / 32; ++w) {
-      const uint32_t t = warp_total[w];
-      warp_off += w < warp ? t : 0u;
-      total += t;
+      for (int w = 0; w < kIdsThreads / 32; ++w) {
+        const uint32_t t = warp_total[k & 1][w];
+        warp_off += w < warp ? t : 0u;
+        total += t;
+      }
     }
-    // number of stage-3 bytes in all earlier ranges
-    if (warp == 0) {
-      uint32_t prefix = 0;
-      if (ranges > 1) {
-        if (lane == 0) atomicExch(state + range, (range == 0 ? kIdsPrefixKnown : kIdsOwnCount) | total);
-        int spins = 0;
-        bool found = false;
-        for (int p0 = range - 1; p0 >= 0 && !found; ) {
-          // four windows of 32 predecessors, nearest first; their loads are independent
-          unsigned long long w[4];
+    // 3. the count of this range is published; the look-back of the range before it is started
+    unsigned long long win[8];
+    if (warp == 0 && ranges > 1) {
+      if (cur && lane == 0) atomicExch(state + range, (range == 0 ? kIdsPrefixKnown : kIdsOwnCount) | total);
+      if (prev > 0) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int p = p0 - 32 * u - lane;
-            w[u] = p >= 0 ? ld_relaxed_u64(state + p) : kIdsPrefixKnown;
+        for (int u = 0; u < 8; ++u) {
+          const int p = prev - 1 - 32 * u - lane;
+          win[u] = p >= 0 ? ld_relaxed_u64(state + p) : kIdsPrefixKnown;
+        }
+      }
+    }
+    const uint32_t* const pseg = bitmap + (((k + 1) & 1) * (kIdsThreads / 32) + warp) * (kIdsMaxRows * 16) + lane * words;
+    const bool fits = prev_total <= (uint32_t)kIdsStageCap;
+    if (prev >= 0 && fits) {
+      // One loop for all the lane's words, from its last bit down to its first: a lane whose word has run out fetches
+      // the one before it while the others go on with theirs, so the lanes of a warp wait for one another once per
+      // range, not once per word.  Every lane makes the same number of turns (the largest need among them), which
+      // keeps the warp together; the body has no branch.
+      uint16_t* dst = staged + prev_local + prev_mine;                         // one past the lane's last position
+      uint32_t top = warp_first + (uint32_t)(lane * words + words) * 32u - 1u;   // position of bit 31 of the word in hand
+      const uint32_t* wp = pseg + words - 1;
+      uint32_t r = *wp;
+#pragma unroll 2
+      for (uint32_t turn = 0; turn < prev_turns; ++turn) {
+        const bool fetch = r == 0u && wp > pseg;
+        wp -= fetch ? 1 : 0;
+        top -= fetch ? 32u : 0u;
+        if (fetch) r = *wp;
+        const uint32_t z = (uint32_t)__clz((int)r);   // 32 for an empty word: nothing is written then
+        const bool emit = r != 0u;
+        dst -= emit ? 1 : 0;
+        if (emit) *dst = (uint16_t)(top - z);
+        r &= ~shr_clamped(0x80000000u, z);             // a shift by 32 gives zero: an empty word stays empty
+      }
+    }
+    if (warp == 0 && prev >= 0) {
+      // number of stage-3 bytes in all ranges before `prev`: windows of 256 predecessors, nearest first, the first
+      // window loaded above
+      uint32_t prefix = 0;
+      if (prev > 0) {
+        int spins = 0;
+        bool found = false, loaded = true;
+        for (int p0 = prev - 1; p0 >= 0 && !found; ) {
+          if (!loaded) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int p = p0 - 32 * u - lane;
+              win[u] = p >= 0 ? ld_relaxed_u64(state + p) : kIdsPrefixKnown;
+            }
           }
-          const bool mine_ready = (w[0] >> 32) != 0ull && (w[1] >> 32) != 0ull && (w[2] >> 32) != 0ull && (w[3] >> 32) != 0ull;
-          if (!__all_sync(0xFFFFFFFFu, mine_ready)) {
+          loaded = false;
+          bool ready = true;
+#pragma unroll
+          for (int u = 0; u < 8; ++u) ready = ready && (win[u] >> 32) != 0ull;
+          if (!__all_sync(0xFFFFFFFFu, ready)) {
             if (++spins > kIdsSpinLimit) {   // cannot happen with tickets in launch order; give up rather than hang
               if (lane == 0) atomicOr(dev_status, 2u);
               break;
@@ -1178,54 +1306,59 @@ takeover_ids_kernel(const uint8_t* __restrict__ stage, int64_t Nc, int Q, int ra
             continue;
           }
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
+          for (int u = 0; u < 8; ++u) {
             if (found) continue;
-            const uint32_t known = __ballot_sync(0xFFFFFFFFu, (w[u] >> 32) == 2ull);
+            const uint32_t known = __ballot_sync(0xFFFFFFFFu, (win[u] >> 32) == 2ull);
             const int stop = known ? __ffs((int)known) - 1 : 31;   // nearest predecessor whose prefix is known
-            uint32_t v = lane <= stop ? (uint32_t)w[u] : 0u;
+            uint32_t v = lane <= stop ? (uint32_t)win[u] : 0u;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
             prefix += v;
             found = known != 0u;
           }
-          p0 -= 128;
+          p0 -= 256;
         }
-        if (lane == 0 && range > 0) atomicExch(state + range, kIdsPrefixKnown | (unsigned long long)(prefix + total));
+        if (lane == 0) atomicExch(state + prev, kIdsPrefixKnown | (unsigned long long)(prefix + prev_total));
       }
       if (lane == 0) {
         prefix_sh = prefix;
-        if (range == ranges - 1 && count != nullptr) *count = prefix + total;
+        if (prev == ranges - 1 && count != nullptr) *count = prefix + prev_total;
       }
     }
     __syncthreads();
-    // positions, row by row: a row's positions are consecutive in the output
-    int64_t row_pos = (int64_t)prefix_sh + warp_off;
-#pragma unroll
-    for (int q = 0; q < kIdsMaxRows; ++q) {
-      if (q < Q) {
-        const uint32_t mm = (m[q >> 1] >> (16 * (q & 1))) & 0xFFFFu;
-        uint32_t incl = (uint32_t)__popc(mm);
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (lane >= o) incl += up;
-        }
-        const int64_t pos = row_pos + incl - (uint32_t)__popc(mm);
-        const int32_t first = (int32_t)(warp_base + q * 512 + lane * 16) - 1;
-        int32_t* dst_id = ids + pos;
-        if (pos + 16 <= ids_cap) {   // the usual case: no bounds test per position
-          for (uint32_t r = mm; r != 0u; r &= r - 1u) *dst_id++ = first + __ffs((int)r);
+    if (prev >= 0) {
+      const int64_t prefix = prefix_sh;
+      const int64_t prev_base = prev * range_bytes - head;   // input position of the range's first byte
+      if (fits) {
+        // 4. a warp instruction writes 32 consecutive positions
+        const int32_t id0 = (int32_t)prev_base;
+        int32_t* const out = ids + prefix;
+        if (prefix + (int64_t)prev_total <= ids_cap) {
+#pragma unroll 4
+          for (uint32_t t = threadIdx.x; t < prev_total; t += kIdsThreads) out[t] = id0 + (int32_t)staged[t];
         } else {
-          int64_t at = pos;
-          for (uint32_t r = mm; r != 0u; r &= r - 1u, ++at)
-            if (at < ids_cap) ids[at] = first + __ffs((int)r);
+          for (uint32_t t = threadIdx.x; t < prev_total; t += kIdsThreads)
+            if (prefix + t < ids_cap) out[t] = id0 + (int32_t)staged[t];
         }
-        row_pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      } else {
+        int64_t at = prefix + prev_local;
+        int64_t first = prev_base + warp_first + (int64_t)(lane * words) * 32;
+        for (int i = 0; i < words; ++i, first += 32)
+          for (uint32_t r = pseg[i]; r != 0u; r &= r - 1u, ++at)
+            if (at < ids_cap) ids[at] = (int32_t)(first + __ffs((int)r) - 1);
       }
     }
-    if (ranges == 1) return;
-    __syncthreads();   // every thread is done with the shared words of this round
+    prev = cur ? range : -1;
+    prev_local = warp_off + incl - mine;   // place of the lane's first position among the range's
+    prev_mine = mine;
+    prev_turns = turns;
+    prev_total = total;
+    range = next;
+    // No barrier here: the next turn writes the other half of the bit map and meets a barrier before it touches the
+    // staging area or the shared words that this turn has read.
+    __syncwarp();
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------------

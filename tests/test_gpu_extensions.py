@@ -187,10 +187,12 @@ def test_vocabulary_sliced_scoring_equals_the_full_definition(M, d, V, cuts):
 @pytest.mark.parametrize("Nc", [0, 1, 15, 16, 4095, 4096, 4097, 70001, (1 << 20) + 5])
 def test_takeover_ids_bit_exact(Nc):
     """Positions of the samples the target takes over and the budget B, against the oracle: random stages, all stage 3,
-    none, an output too short for all of them, and a stage array that is not 16-byte aligned."""
+    none, arbitrary byte values, an output too short for all of them, and a stage array that is not 16-byte aligned."""
     rng = np.random.default_rng(Nc + 1)
     cases = [rng.choice(np.array([1, 2, 3], np.uint8), size=Nc, p=[0.05, 0.7, 0.25]),
-             np.full(Nc, 3, np.uint8), np.full(Nc, 2, np.uint8)]
+             np.full(Nc, 3, np.uint8), np.full(Nc, 2, np.uint8),
+             # every byte value, threes made frequent: only the byte 3 itself counts (0x83, 0x13, 0x02, 0x07 do not)
+             np.where(rng.random(Nc) < 0.3, 3, rng.integers(0, 256, Nc)).astype(np.uint8)]
     ws = workspace(binding.takeover_ids_workspace_bytes(Nc))
     for stage_h in cases:
         want = orc.takeover_ids(stage_h) if Nc < 200000 else np.flatnonzero(stage_h == 3).astype(np.int32)
