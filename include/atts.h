@@ -236,13 +236,18 @@ int atts_classify_threshold(const float* scores, int64_t Nc, const float* tau, u
  * input group_ids[j].  Reading adopted: the same count as the marginal form over the group's scores,
  *   numer[j] = 1 + #{ i in group : calib[i] >= scores[j] },  denom[j] = |group| + 1,  p = numer / denom.
  *   scores        dev  [Nc] fp32;  group_ids dev [Nc] int32 in [0, G) (outside: ATTS_DEV_GROUP_ID_RANGE, numer 0)
- *   calib_segments dev fp32: the groups' scores one after the other, each group ascending (NaNs last)
- *   seg_offsets   dev  [G + 1] int32, group g is calib_segments[seg_offsets[g] .. seg_offsets[g+1])
+ *   calib_segments dev [calib_total] fp32: the groups' scores one after the other, each group ascending (NaNs last)
+ *   calib_total   number of entries of calib_segments, < 2^31
+ *   seg_offsets   dev  [G + 1] int32, group g is calib_segments[seg_offsets[g] .. seg_offsets[g+1]); a group whose
+ *                      offsets are not 0 <= seg_offsets[g] <= seg_offsets[g+1] <= calib_total is never read: its
+ *                      candidates get numer 0 and ATTS_DEV_GROUP_ID_RANGE is recorded
  *   numer, denom  dev  [Nc] uint32 out;  pvalue dev [Nc] fp32 out, may be NULL
+ * Every array 4-byte aligned; 16-byte aligned scores, group_ids and outputs take 128-bit loads and stores, a 32-byte
+ * aligned calib_segments 256-bit loads.
  */
 int atts_conformal_rank_conditional(const float* scores, const int32_t* group_ids, int64_t Nc,
-                                    const float* calib_segments, const int32_t* seg_offsets, int64_t G,
-                                    uint32_t* numer, uint32_t* denom, float* pvalue, void* cuda_stream);
+                                    const float* calib_segments, int64_t calib_total, const int32_t* seg_offsets,
+                                    int64_t G, uint32_t* numer, uint32_t* denom, float* pvalue, void* cuda_stream);
 
 /*
  * atts_classify with every candidate's own denominator: reject iff 1 <= numer <= floor(alpha * denom)

@@ -68,8 +68,8 @@ def load(rebuild_if_stale: bool = True) -> ctypes.CDLL:
     lib.atts_rms_inv.argtypes = [c_void_p, c_int64, c_int64, ctypes.c_float, c_void_p, c_void_p]
     lib.atts_threshold.argtypes = [c_void_p, c_int64, c_double, c_void_p, c_void_p]
     lib.atts_classify_threshold.argtypes = [c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
-    lib.atts_conformal_rank_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_void_p,
-                                                    c_void_p, c_void_p, c_void_p]
+    lib.atts_conformal_rank_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_int64, c_void_p, c_int64,
+                                                    c_void_p, c_void_p, c_void_p, c_void_p]
     lib.atts_classify_conditional.argtypes = [c_void_p, c_void_p, c_int64, c_double, c_void_p, c_void_p, c_void_p]
     lib.atts_debug_score_plan.argtypes = [c_int64, c_int64, c_int64, c_int32, c_int32, POINTER(c_int32)]
     lib.atts_debug_score_unit.argtypes = [c_int64, c_int64, c_int64, c_int32, c_int32, c_int32, POINTER(c_int32)]
@@ -199,8 +199,9 @@ def takeover_ids(stage, ids, count, workspace) -> None:
 def conformal_rank_conditional(scores, group_ids, calib_segments, seg_offsets, numer, denom, pvalue=None) -> None:
     """Rank each score against the ascending calibration segment of its own group."""
     _check(load().atts_conformal_rank_conditional(_ptr(scores), _ptr(group_ids), scores.numel(), _ptr(calib_segments),
-                                                  _ptr(seg_offsets), seg_offsets.numel() - 1, _ptr(numer), _ptr(denom),
-                                                  _ptr(pvalue), _stream()), "atts_conformal_rank_conditional")
+                                                  calib_segments.numel(), _ptr(seg_offsets), seg_offsets.numel() - 1,
+                                                  _ptr(numer), _ptr(denom), _ptr(pvalue), _stream()),
+           "atts_conformal_rank_conditional")
 
 
 def classify_conditional(numer, denom, alpha: float, stage, stage_counts=None) -> None:

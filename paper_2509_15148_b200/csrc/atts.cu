@@ -626,10 +626,12 @@ int atts_takeover_ids(const uint8_t* stage, int64_t Nc, int32_t* ids, int64_t id
 }
 
 int atts_conformal_rank_conditional(const float* scores, const int32_t* group_ids, int64_t Nc, const float* calib_segments,
-                                    const int32_t* seg_offsets, int64_t G, uint32_t* numer, uint32_t* denom, float* pvalue,
-                                    void* cuda_stream) {
-  if (Nc < 0 || Nc >= (1ll << 31) || G < 0 || G >= (1ll << 31)) return ATTS_ERR_SHAPE;
+                                    int64_t calib_total, const int32_t* seg_offsets, int64_t G, uint32_t* numer,
+                                    uint32_t* denom, float* pvalue, void* cuda_stream) {
+  if (Nc < 0 || Nc >= (1ll << 31) || G < 0 || G >= (1ll << 31) || calib_total < 0 || calib_total >= (1ll << 31))
+    return ATTS_ERR_SHAPE;
   if (Nc > 0 && (!scores || !group_ids || !numer || !denom || !seg_offsets)) return ATTS_ERR_NULL;
+  if (Nc > 0 && calib_total > 0 && !calib_segments) return ATTS_ERR_NULL;
   if (!aligned(scores, 4) || !aligned(group_ids, 4) || !aligned(numer, 4) || !aligned(denom, 4) || !aligned(pvalue, 4) ||
       !aligned(calib_segments, 4) || !aligned(seg_offsets, 4))
     return ATTS_ERR_ALIGN;
@@ -642,7 +644,8 @@ int atts_conformal_rank_conditional(const float* scores, const int32_t* group_id
   const bool vec4 = aligned(scores, 16) && aligned(group_ids, 16) && aligned(numer, 16) && aligned(denom, 16) &&
                     aligned(pvalue, 16);
   rank_conditional_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
-      scores, group_ids, Nc, calib_segments, seg_offsets, (int)G, numer, denom, pvalue, vec4, di->dev_status);
+      scores, group_ids, Nc, calib_segments, (int)calib_total, seg_offsets, (int)G, numer, denom, pvalue, vec4,
+      aligned(calib_segments, 32), di->dev_status);
   return launch_status();
 }
 

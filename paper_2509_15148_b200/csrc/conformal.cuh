@@ -1363,22 +1363,24 @@ takeover_ids_kernel(const uint8_t* __restrict__ base, int64_t len, int head, int
 
 // ---------------------------------------------------------------------------------------------
 // Conditional coverage (Proposition 2): a candidate is ranked against the calibration scores of its own
-// input only.  The per-input buffers are ascending segments of one array; segments are short (the m samples
-// of one input), so a thread searches its segment directly in (L2-resident) global memory.
+// input only.  The per-input buffers are ascending segments of one array.
 //   numer = 1 + #{own segment >= s},  denom = |segment| + 1,  p = numer / denom;  reject iff
 //   1 <= numer <= floor(alpha * denom)  (evaluated in IEEE double, as on the host for the marginal form).
+// When the candidates of one input arrive together a warp stages the few segments it needs in shared memory.
+// When they do not, every load of a search is a 32-byte sector of its own from L2, and those sectors are what
+// bounds the kernel; the search is then made over the aligned groups of eight entries that overlap the segment
+// (one probe per step, at a group's last entry) and finished with a single 32-byte load of the group found.
 // ---------------------------------------------------------------------------------------------
 constexpr int kCondStage = 512;   // calibration entries a warp can stage in shared memory (2 KB)
 
-// Lower bound of four scores in their own segments [lo, lo + len), advanced together so that the dependent loads
-// overlap; `data` is indexed by the same positions as the segments (shared or global memory).
-template <bool GLOBAL>
+// Lower bound of four scores in their own segments [lo, lo + len) of `data` (shared memory), advanced together so
+// that the dependent loads overlap.
 __device__ __forceinline__ void lower_bound_four(const float* data, const float (&s)[4], int (&lo)[4], int (&len)[4]) {
   const float qnan = __uint_as_float(0x7FC00000u);
   while (max(max(len[0], len[1]), max(len[2], len[3])) > 0) {
     float v[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = len[e] > 0 ? (GLOBAL ? __ldg(data + lo[e] + (len[e] >> 1)) : data[lo[e] + (len[e] >> 1)]) : qnan;
+    for (int e = 0; e < 4; ++e) v[e] = len[e] > 0 ? data[lo[e] + (len[e] >> 1)] : qnan;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       if (len[e] > 0) {
@@ -1391,11 +1393,73 @@ __device__ __forceinline__ void lower_bound_four(const float* data, const float 
   }
 }
 
-__global__ void __launch_bounds__(256)
+// The same in global memory, for segments [lo, end) with len = end - lo entries (len <= 0: nothing to search).
+// Group g is calib[8 g, 8 g + 8).  All entries of a group whose last entry is below s are below s, and none of a
+// group after one whose last entry is not: the first group of the segment whose last entry is not below s (the
+// segment's last group if there is none) holds the boundary.  It is found by bisection over the groups, one probe a
+// step, and read whole with one 32-byte load (`vec8`: calib is 32-byte aligned; `total` entries exist).
+__device__ __forceinline__ void lower_bound_four_global(const float* __restrict__ calib, int total, bool vec8,
+                                                        const float (&s)[4], int (&lo)[4], const int (&end)[4],
+                                                        const int (&len)[4]) {
+  const float qnan = __uint_as_float(0x7FC00000u);
+  int g[4], gn[4];   // the boundary group is in [g, g + gn]
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    g[e] = lo[e] >> 3;
+    gn[e] = len[e] > 0 ? ((end[e] - 1) >> 3) - g[e] : 0;
+  }
+  while (max(max(gn[0], gn[1]), max(gn[2], gn[3])) > 0) {
+    float v[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = gn[e] > 0 ? __ldg(calib + 8 * (g[e] + (gn[e] >> 1)) + 7) : qnan;   // inside the segment
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (gn[e] > 0) {
+        const int half = gn[e] >> 1;
+        const bool less = v[e] < s[e];
+        g[e] = less ? g[e] + half + 1 : g[e];
+        gn[e] = less ? gn[e] - half - 1 : half;
+      }
+    }
+  }
+  // two candidates at a time: sixteen registers of loaded entries instead of thirty-two
+#pragma unroll
+  for (int h = 0; h < 4; h += 2) {
+    float w[2][8];
+#pragma unroll
+    for (int e = h; e < h + 2; ++e) {
+      const int g0 = 8 * g[e];
+      if (len[e] > 0 && vec8 && g0 + 8 <= total) {
+        asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=f"(w[e - h][0]), "=f"(w[e - h][1]), "=f"(w[e - h][2]), "=f"(w[e - h][3]), "=f"(w[e - h][4]),
+                       "=f"(w[e - h][5]), "=f"(w[e - h][6]), "=f"(w[e - h][7])
+                     : "l"(calib + g0));
+      } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          w[e - h][i] = (len[e] > 0 && g0 + i >= lo[e] && g0 + i < end[e]) ? __ldg(calib + g0 + i) : qnan;
+      }
+    }
+#pragma unroll
+    for (int e = h; e < h + 2; ++e) {
+      if (len[e] > 0) {
+        const int g0 = 8 * g[e];
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) c += (g0 + i >= lo[e] && g0 + i < end[e] && w[e - h][i] < s[e]) ? 1 : 0;
+        lo[e] = max(g0, lo[e]) + c;
+      }
+    }
+  }
+}
+
+// total: entries of calib that exist.  A group whose offsets do not describe a part of them (negative, beyond
+// total, or decreasing) is treated like a group id out of range: flagged, and its candidates get no score.
+__global__ void __launch_bounds__(256, 5)
 rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restrict__ group_ids, int64_t Nc,
-                        const float* __restrict__ calib, const int32_t* __restrict__ seg_offsets, int G,
+                        const float* __restrict__ calib, int total, const int32_t* __restrict__ seg_offsets, int G,
                         uint32_t* __restrict__ numer, uint32_t* __restrict__ denom, float* __restrict__ pvalue,
-                        bool vec4, unsigned int* __restrict__ dev_status) {
+                        bool vec4, bool vec8, unsigned int* __restrict__ dev_status) {
   // A warp takes 128 consecutive candidates, four per lane (128-bit loads and stores when every array is 16-byte
   // aligned: vec4).  The candidates of one input usually arrive together, so the segments a warp needs are few
   // and adjacent: if they span at most kCondStage entries the warp copies that span into shared memory with
@@ -1428,9 +1492,11 @@ rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restr
     int span_lo = 0x7FFFFFFF, span_hi = 0;
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const bool ok = g[e] >= 0 && g[e] < G;
+      bool ok = g[e] >= 0 && g[e] < G;
+      int a = ok ? __ldg(seg_offsets + g[e]) : 0, b = ok ? __ldg(seg_offsets + g[e] + 1) : 0;
+      ok = ok && a >= 0 && a <= b && b <= total;
+      if (!ok) a = b = 0;
       bad = bad || (!ok && j + e < Nc);
-      const int a = ok ? __ldg(seg_offsets + g[e]) : 0, b = ok ? __ldg(seg_offsets + g[e] + 1) : 0;
       lo[e] = a;
       end[e] = b;
       den[e] = ok ? (uint32_t)(b - a) + 1u : 1u;
@@ -1440,7 +1506,7 @@ rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restr
         span_hi = max(span_hi, b);
       }
     }
-    if (bad) atomicOr(dev_status, 4u);  // group id out of range: no calibration set, treated as "no score"
+    if (bad) atomicOr(dev_status, 4u);  // no such group, or not a part of the calibration array: no score
     const bool scored[4] = {len[0] >= 0, len[1] >= 0, len[2] >= 0, len[3] >= 0};
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -1452,9 +1518,9 @@ rank_conditional_kernel(const float* __restrict__ scores, const int32_t* __restr
       __syncwarp();                          // the previous round's searches are done with the staging area
       for (int t = span_lo + lane; t < span_hi; t += 32) stage[t - span_lo] = __ldg(calib + t);
       __syncwarp();
-      lower_bound_four<false>(stage - span_lo, s, lo, len);
+      lower_bound_four(stage - span_lo, s, lo, len);
     } else {
-      lower_bound_four<true>(calib, s, lo, len);
+      lower_bound_four_global(calib, total, vec8, s, lo, end, len);
     }
     uint32_t num[4];
     float p[4];

@@ -75,6 +75,27 @@ def test_conditional_rank_and_classify_bit_exact():
     binding.conformal_rank_conditional(dev(scores), dev(gid2), dev(calib), dev(off), numer, denom, None)
     assert binding.last_device_status() & binding.DEV_GROUP_ID_RANGE
     assert host_u32(numer)[10] == 0
+    # a calibration array that is not 32-byte aligned (no 256-bit loads), with candidates in random and in grouped order
+    shifted = dev(np.concatenate([np.zeros(1, np.float32), calib]))[1:]
+    for order in (np.arange(Nc), np.argsort(gid, kind="stable")):
+        binding.conformal_rank_conditional(dev(scores[order]), dev(gid[order]), shifted, dev(off), numer, denom, None)
+        assert np.array_equal(host_u32(numer), want_numer[order])
+    binding.conformal_rank_conditional(dev(scores[order]), dev(gid[order]), dev(calib), dev(off), numer, denom, None)
+    assert np.array_equal(host_u32(numer), want_numer[order])
+    # offsets that do not describe a part of the calibration array (decreasing, negative, beyond its end) are
+    # flagged like a bad group id and never used as addresses; the other groups are unaffected
+    for g_bad, (a, b) in ((7, (int(off[8]) + 5, int(off[8]))), (9, (-4, int(off[10]))), (G - 1, (int(off[G - 1]), int(off[G]) + 1000))):
+        off2 = off.copy()
+        if g_bad == G - 1:
+            off2[G] = b
+        else:
+            off2[g_bad] = a
+        hit = (gid == g_bad) | ((gid == g_bad - 1) if g_bad != G - 1 else False)
+        binding.conformal_rank_conditional(dev(scores), dev(gid), dev(calib), dev(off2), numer, denom, None)
+        assert binding.last_device_status() & binding.DEV_GROUP_ID_RANGE
+        got = host_u32(numer)
+        assert np.array_equal(got[~hit], want_numer[~hit])
+        assert np.all(got[gid == g_bad] == 0)
     # ragged tails and arrays that are not 16-byte aligned take the scalar loads and stores
     for start, stop in ((0, Nc - 1), (1, Nc), (3, Nc - 2), (0, 3)):
         m = stop - start
