@@ -100,11 +100,11 @@ static int device_info(const DeviceInfo** out) {
       ok = ok && cudaFuncSetAttribute(rank_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, rank_smem) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 << kIndexMaxTreeLog2) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 << kIndexMaxTreeLog2) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 << kIndexMaxTreeLog2) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 << kIndexMaxTreeLog2) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(rank_indexed_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 << kIndexMaxTreeLog2) == cudaSuccess;
       const int bucket_smem = 4 * ((1 << kBucketMaxLog2) + 1 + 2 * kBucketMaxN + kBucketPad + 2);
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(rank_bucket_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, bucket_smem) == cudaSuccess;

@@ -471,7 +471,8 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
 //           implicit search tree in breadth-first order, ready to be copied into shared memory.
 // A candidate descends the tree (P shared-memory steps) to its group of G, then narrows by a factor of 8 per
 // 32-byte load: A loads of aux entries and one of the buffer.  A is the smallest number of levels for which the
-// tree has at most 8191 nodes: 0 for n < 65,528, 1 up to 524,223, 2 up to 4,193,791, 3 beyond.
+// tree has at most 8191 nodes: 0 for n < 65,528, 1 up to 524,223, 2 up to 4,193,791; beyond that a tree of up to
+// 32767 nodes with two levels (n up to 16,776,703) and only then a third level.
 //
 // Two slots.  An update reads the buffer copy of the slot that describes the present fill n and writes the merged
 // buffer to the other slot and to the caller's buffer, together with the other slot's aux entries and tree: no
@@ -484,7 +485,8 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
 //   aux_1, aux_2, aux_3, buf (every array a multiple of 8 words long).
 // ---------------------------------------------------------------------------------------------
 constexpr int kIndexHeaderWords = 64;
-constexpr int kIndexTreeWords = 1 << kRankMaxTableLog2;               // 8191 nodes + 1 pad
+constexpr int kIndexMaxTreeLog2 = 15;                                 // the largest tree: 32767 nodes (128 KB of shared memory)
+constexpr int kIndexTreeWords = 1 << kIndexMaxTreeLog2;
 constexpr int kIndexMaxLevels = 3;
 constexpr int kIndexCountScratch = 32;   // header words [32, 45): stage-count accumulators of the rank kernel, block counter
 constexpr uint32_t kIndexMagic = 0x41545832u;
@@ -519,6 +521,8 @@ __host__ __device__ inline IndexShape index_shape(int64_t n) {
   IndexShape s;
   s.A = 0;
   while ((n >> (3 * (s.A + 1))) + 1 > (1 << kRankMaxTableLog2) - 1) ++s.A;
+  // a third aux level costs every candidate a fourth load from L2: a deeper tree is cheaper while it still fits
+  if (s.A == kIndexMaxLevels && (n >> (3 * kIndexMaxLevels)) + 1 <= (1 << kIndexMaxTreeLog2) - 1) --s.A;
   s.ns = (int)(n >> (3 * (s.A + 1))) + 1;
   s.P = 1;
   while ((1 << s.P) - 1 < s.ns) ++s.P;
@@ -702,7 +706,9 @@ rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, int n, uint32_
       case 10: rank_four_indexed<10>(s, sp, A, aux, calib, n, r); break;
       case 11: rank_four_indexed<11>(s, sp, A, aux, calib, n, r); break;
       case 12: rank_four_indexed<12>(s, sp, A, aux, calib, n, r); break;
-      default: rank_four_indexed<13>(s, sp, A, aux, calib, n, r); break;
+      case 13: rank_four_indexed<13>(s, sp, A, aux, calib, n, r); break;
+      case 14: rank_four_indexed<14>(s, sp, A, aux, calib, n, r); break;
+      default: rank_four_indexed<15>(s, sp, A, aux, calib, n, r); break;
     }
     float p[4] = {qnan, qnan, qnan, qnan};
     if (pvalue) {
