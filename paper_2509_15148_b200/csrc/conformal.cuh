@@ -1271,12 +1271,14 @@ takeover_ids_kernel(const uint8_t* __restrict__ base, int64_t len, int head, int
       uint32_t top = warp_first + (uint32_t)(lane * words + words) * 32u - 1u;   // position of bit 31 of the word in hand
       const uint32_t* wp = pseg + words - 1;
       uint32_t r = *wp;
+      uint32_t ahead = wp > pseg ? wp[-1] : 0u;   // the word before the one in hand, loaded before it is needed
 #pragma unroll 2
       for (uint32_t turn = 0; turn < prev_turns; ++turn) {
         const bool fetch = r == 0u && wp > pseg;
         wp -= fetch ? 1 : 0;
         top -= fetch ? 32u : 0u;
-        if (fetch) r = *wp;
+        r = fetch ? ahead : r;
+        if (fetch && wp > pseg) ahead = wp[-1];
         const uint32_t z = (uint32_t)__clz((int)r);   // 32 for an empty word: nothing is written then
         const bool emit = r != 0u;
         dst -= emit ? 1 : 0;
