@@ -39,7 +39,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 KERNELS_PER_STEP = 6  # lmhead_lse, lse_combine, segment_score, rank, classify, small_update (n + k small: one block)
 # DRAM bytes per launch of the fused kernel on this workload, from an ncu capture (profiles/), valid only for
 # the kernel source it was taken on: (sha256 of csrc/lmhead_lse.cuh, dram__bytes_read.sum + dram__bytes_write.sum).
-K1_TRAFFIC = ("18fa410ba28afbe3a4a16a57cdf0e525b99c7545f56f72480992126599fc958b", 5.255e10)
+K1_TRAFFIC = ("63ed8c15ce1c5157e25ce877a7cba86bd55c145fefd26b445bb2b96233c252f6", 8.680e10)
 
 
 def k1_traffic_bytes():
@@ -849,7 +849,7 @@ def run_ours(args):
                      "traffic": k1_traffic_bytes() if args.workload == WORKLOAD else None,
                      "traffic_note": "stored figure: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of "
                                      "this kernel source on this workload (mean of 3 launches), not measured in this run; "
-                                     "captures on other boxes ranged 45-98 GB per launch; null once the kernel source changes"},
+                                     "captures on other boxes and builds ranged 45-105 GB per launch; null once the kernel source changes"},
         "stage_counts_last_step": stage_counts_last, "calib_n_end": state["n"],
     }
     # Asynchronous arithmetic intensity of the step (the paper's r = T_c / (T_m + T_s)): T_c the fused kernel's time,
