@@ -659,16 +659,27 @@ rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, int n, uint32_
                     uint32_t* __restrict__ numer, float* __restrict__ pvalue, const FusedClassify fc,
                     unsigned int* __restrict__ dev_status) {
   extern __shared__ float sp[];
+  const float qnan = __uint_as_float(0x7FC00000u);
+  const int64_t quads = (Nc + 3) >> 2;
+  const int64_t share = (quads + gridDim.x - 1) / gridDim.x;
+  const int64_t q_end = min(quads, ((int64_t)blockIdx.x + 1) * share);
+  const int64_t q_first = (int64_t)blockIdx.x * share + threadIdx.x;
   pdl_launch_dependents();
   pdl_wait();   // everything read below may come from the kernel before this one
-  // an index that does not describe this fill of the buffer would give wrong ranks silently: refuse it
-  const uint32_t cap = index[1];   // the capacity the index was laid out for, as its builder recorded it
-  const int slot = index_find(index, cap, (uint32_t)n);
+  // the thread's first four scores are on their way while the index is looked at and the table filled
+  float4 nxt = make_float4(qnan, qnan, qnan, qnan);
+  if (q_first < q_end && 4 * q_first + 4 <= Nc) nxt = *reinterpret_cast<const float4*>(scores + 4 * q_first);
+  // an index that does not describe this fill of the buffer would give wrong ranks silently: refuse it.  The header
+  // words that matter (magic and capacity, the two slots' descriptions) are read together, in one round trip.
+  const uint4 h0 = *reinterpret_cast<const uint4*>(index), d0 = *reinterpret_cast<const uint4*>(index + 8),
+              d1 = *reinterpret_cast<const uint4*>(index + 16);
+  const uint32_t cap = h0.y;   // the capacity the index was laid out for, as its builder recorded it
+  const int slot = h0.x != kIndexMagic ? -1 : (d0.x == (uint32_t)n ? 0 : (d1.x == (uint32_t)n ? 1 : -1));
   if (slot < 0) {
     if (threadIdx.x == 0 && blockIdx.x == 0) atomicOr(dev_status, 8u);
     return;
   }
-  const int P = (int)index[8 + 8 * slot + 1], A = (int)index[8 + 8 * slot + 2];
+  const int P = (int)(slot ? d1.y : d0.y), A = (int)(slot ? d1.z : d0.z);
   const IndexLayout L = index_layout(cap);
   const float* const base = reinterpret_cast<const float*>(index + kIndexHeaderWords + (size_t)slot * L.slot_words);
   const float* const aux[kIndexMaxLevels] = {base + L.aux_off[0], base + L.aux_off[1], base + L.aux_off[2]};
@@ -677,22 +688,17 @@ rank_indexed_kernel(const float* __restrict__ scores, int64_t Nc, int n, uint32_
   __syncthreads();
   StageTally<NA> tally;
   const float denom = (float)(n + 1);
-  const float qnan = __uint_as_float(0x7FC00000u);
-  const int64_t quads = (Nc + 3) >> 2;
-  const int64_t share = (quads + gridDim.x - 1) / gridDim.x;
-  const int64_t q_end = min(quads, ((int64_t)blockIdx.x + 1) * share);
-  for (int64_t q = (int64_t)blockIdx.x * share + threadIdx.x; q < q_end; q += kRankThreads) {
+  for (int64_t q = q_first; q < q_end; q += kRankThreads) {
     const int64_t j = 4 * q;
-    float s[4];
+    float s[4] = {nxt.x, nxt.y, nxt.z, nxt.w};
     uint32_t r[4];
     const bool full = j + kRankPerThread <= Nc;
-    if (full) {
-      const float4 s4 = *reinterpret_cast<const float4*>(scores + j);
-      s[0] = s4.x; s[1] = s4.y; s[2] = s4.z; s[3] = s4.w;
-    } else {
+    if (!full) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) s[e] = (j + e < Nc) ? scores[j + e] : qnan;
     }
+    if (q + kRankThreads < q_end && j + 4 * kRankThreads + 4 <= Nc)   // the scores of the next round
+      nxt = *reinterpret_cast<const float4*>(scores + j + 4 * kRankThreads);
     switch (P) {
       case 1: rank_four_indexed<1>(s, sp, A, aux, calib, n, r); break;
       case 2: rank_four_indexed<2>(s, sp, A, aux, calib, n, r); break;
