@@ -71,8 +71,10 @@ int atts_version(void);
 int atts_score_workspace_bytes(int64_t M, int64_t d, int64_t V, int64_t S, size_t* bytes);
 
 /*
- * Target-model scoring of draft tokens (Sec. 3.3 "Verification"; the score of Sec. 3.2,
- * s = -l with l the negative log-likelihood loss of Eq. 2).
+ * Target-model scoring of draft tokens (Sec. 3.3 "Verification"; the score of Sec. 3.2, the equation before
+ * Eq. p-value).  Reading adopted: the score handed to the conformal layer is the sample's mean negative
+ * log-likelihood under the target model (larger = the target finds the draft less likely), so that p <= alpha
+ * rejects the unlikely samples; score modes 2 and 3 give the opposite sign.
  *
  * For every row i (one scored draft token): logits z_i = W h_i over the whole vocabulary,
  * token_logprob[i] = z_i[token_ids[i]] - log sum_v exp(z_i[v]).  The logits are produced tile by
@@ -152,12 +154,13 @@ int atts_rms_inv(const void* hidden_bf16, int64_t M, int64_t d, float eps, float
  * Ties count.  A NaN calibration score (sorted last) counts for every candidate; a NaN candidate
  * has no score: numer = 0, pvalue = NaN.
  *
- *   scores        dev  [Nc] fp32
+ *   scores        dev  [Nc] fp32, 16-byte aligned
  *   calib_sorted  dev  [n] fp32 ascending, NaNs last (as atts_calib_update leaves it); may be NULL
  *                      when n == 0
  *   Nc, n              0 <= Nc < 2^31, 0 <= n < 2^24 - 1 (so that n + 1 is exact in fp32)
- *   numer         dev  [Nc] uint32 out
- *   pvalue        dev  [Nc] fp32 out (one correctly rounded fp32 division), may be NULL
+ *   numer         dev  [Nc] uint32 out, 16-byte aligned
+ *   pvalue        dev  [Nc] fp32 out (one correctly rounded fp32 division), 16-byte aligned, may be NULL
+ * A pointer that is not aligned as stated is refused with ATTS_ERR_ALIGN before anything is launched.
  */
 int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sorted, int64_t n,
                         uint32_t* numer, float* pvalue, void* cuda_stream);
@@ -170,9 +173,9 @@ int atts_conformal_rank(const float* scores, int64_t Nc, const float* calib_sort
  *   1 <= numer <= k_alpha  -> ATTS_STAGE_TARGET    (p <= alpha)
  *   otherwise              -> ATTS_STAGE_ACCEPTED  (p >  alpha)
  *
- *   numer         dev  [Nc] uint32, as written by atts_conformal_rank for the same n
+ *   numer         dev  [Nc] uint32, as written by atts_conformal_rank for the same n, 16-byte aligned
  *   alpha              0 < alpha < 1, else ATTS_ERR_ARG
- *   stage         dev  [Nc] uint8 out
+ *   stage         dev  [Nc] uint8 out, 16-byte aligned (ATTS_ERR_ALIGN otherwise)
  *   stage_counts  dev  [3] uint32 out (numbers of samples in stages 1, 2, 3; the third is the
  *                      budget B of "Budget Prediction"), overwritten; may be NULL
  */

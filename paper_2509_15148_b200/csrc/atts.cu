@@ -18,7 +18,8 @@ namespace atts {
 __device__ unsigned int g_dev_status = 0u;
 
 struct DeviceInfo {
-  bool ready = false;
+  bool ready = false;                 // the probe has run (under the mutex)
+  std::atomic<bool> probed{false};    // set last: a reader that sees it may use every other field without the mutex
   int status = ATTS_OK;  // sticky result of the probe
   int sm_count = 0;
   int pair_workers = 0;  // CTA pairs (clusters of 2) of the fused kernel that can be resident at once; 0 = unusable
@@ -54,8 +55,12 @@ static int device_info(const DeviceInfo** out) {
     cudaGetLastError();
     return ATTS_ERR_CUDA;
   }
-  std::lock_guard<std::mutex> lock(g_mu);
   DeviceInfo& di = g_info[dev];
+  if (di.probed.load(std::memory_order_acquire)) {   // every call after the first on a device: no lock
+    *out = &di;
+    return di.status;
+  }
+  std::lock_guard<std::mutex> lock(g_mu);
   if (!di.ready) {
     di.ready = true;
     int major = 0;
@@ -123,6 +128,7 @@ static int device_info(const DeviceInfo** out) {
       }
     }
   }
+  di.probed.store(true, std::memory_order_release);
   *out = &di;
   return di.status;
 }
@@ -197,7 +203,26 @@ static int check_score_shape(int64_t M, int64_t d, int64_t V, int64_t S) {
   return ATTS_OK;
 }
 
+// A tensor map is a function of the base address, the shape and the box alone, so the last few are kept per host
+// thread: a caller that scores batch after batch from the same buffers pays for the encoding once.
+struct TmapEntry {
+  const void* base = nullptr;
+  int64_t rows = 0, cols = 0;
+  int box_rows = 0;
+  const DeviceInfo* di = nullptr;
+  CUtensorMap map;
+};
 static int encode_2d(const DeviceInfo* di, CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  constexpr int kKept = 8;
+  thread_local TmapEntry kept[kKept];
+  thread_local int next = 0;
+  for (int i = 0; i < kKept; ++i) {
+    const TmapEntry& e = kept[i];
+    if (e.base == base && e.rows == rows && e.cols == cols && e.box_rows == box_rows && e.di == di) {
+      *map = e.map;
+      return ATTS_OK;
+    }
+  }
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
   cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
@@ -205,7 +230,11 @@ static int encode_2d(const DeviceInfo* di, CUtensorMap* map, const void* base, i
   CUresult r = di->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? ATTS_OK : ATTS_ERR_CUDA;
+  if (r != CUDA_SUCCESS) return ATTS_ERR_CUDA;
+  TmapEntry& e = kept[next];
+  next = (next + 1) % kKept;
+  e.base = base; e.rows = rows; e.cols = cols; e.box_rows = box_rows; e.di = di; e.map = *map;
+  return ATTS_OK;
 }
 
 // Built-in scratch of atts_calib_update_static: the merged copy, ATTS_STATIC_MAX_TOTAL f32.  In host code this name is only a handle for
