@@ -1436,12 +1436,12 @@ __device__ __forceinline__ void lower_bound_four_global(const float* __restrict_
       }
     }
   }
-  // two candidates at a time: sixteen registers of loaded entries instead of thirty-two
+  // one candidate at a time: eight registers of loaded entries instead of thirty-two
 #pragma unroll
-  for (int h = 0; h < 4; h += 2) {
-    float w[2][8];
+  for (int h = 0; h < 4; h += 1) {
+    float w[1][8];
 #pragma unroll
-    for (int e = h; e < h + 2; ++e) {
+    for (int e = h; e < h + 1; ++e) {
       const int g0 = 8 * g[e];
       if (len[e] > 0 && vec8 && g0 + 8 <= total) {
         asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
@@ -1455,7 +1455,7 @@ __device__ __forceinline__ void lower_bound_four_global(const float* __restrict_
       }
     }
 #pragma unroll
-    for (int e = h; e < h + 2; ++e) {
+    for (int e = h; e < h + 1; ++e) {
       if (len[e] > 0) {
         const int g0 = 8 * g[e];
         int c = 0;
