@@ -286,14 +286,15 @@ int atts_calib_update(float* calib, int64_t n, int64_t cap, const float* new_sco
  * Ranking many candidates against a buffer too large for shared memory is bound by the divergent loads
  * of each candidate's search.  An index kept beside the buffer - a copy of the buffer, the last entry of every
  * aligned group of 8, 64, ... entries, and the coarsest of those levels laid out as a search tree - lets a
- * candidate finish with one to four 32-byte loads (two up to n = 524,223, three up to 4,193,791).  The index
+ * candidate finish with one to four 32-byte loads (one up to n = 262,143, two up to 2,097,151, three up to
+ * 16,776,703).  The index
  * holds all of this twice: an update reads the half that describes the present fill and writes the other half
  * and the caller's buffer in one pass, so it needs no copy back, and it touches nothing that a rank of the fill
  * it started from reads.  The calibration state of a caller that uses these calls is the buffer AND its index:
  * both describe the same fill n.
  *
  *   atts_calib_index_bytes   host out *bytes: size of an index for buffers of up to `cap` entries,
- *                            0 <= cap < 2^24 - 1 (about 9.2 bytes per entry plus 64 KB)
+ *                            0 <= cap < 2^24 - 1 (about 9.2 bytes per entry plus 256 KB)
  *   index         dev  256-byte aligned; index_bytes: the size of that allocation, the same value in every call
  *                      (the layout is derived from it); too small for n (+ k): ATTS_ERR_WORKSPACE
  *   atts_calib_index_build   makes `index` describe calib_sorted[0, n) (a buffer filled some other way, or the

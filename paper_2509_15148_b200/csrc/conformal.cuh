@@ -471,8 +471,9 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
 //           implicit search tree in breadth-first order, ready to be copied into shared memory.
 // A candidate descends the tree (P shared-memory steps) to its group of G, then narrows by a factor of 8 per
 // 32-byte load: A loads of aux entries and one of the buffer.  A is the smallest number of levels for which the
-// tree has at most 8191 nodes: 0 for n < 65,528, 1 up to 524,223, 2 up to 4,193,791; beyond that a tree of up to
-// 32767 nodes with two levels (n up to 16,776,703) and only then a third level.
+// tree has at most 32767 nodes (128 KB of shared memory; a level more costs every candidate one more load from L2, a
+// deeper tree one more step in shared memory): 0 for n <= 262,143, 1 up to 2,097,151, 2 up to 16,776,703, 3 for the
+// last few hundred sizes of the range.
 //
 // Two slots.  An update reads the buffer copy of the slot that describes the present fill n and writes the merged
 // buffer to the other slot and to the caller's buffer, together with the other slot's aux entries and tree: no
@@ -481,7 +482,7 @@ rank_bucket_kernel(const float* __restrict__ scores, int64_t Nc, const float* __
 //
 // Layout (32-bit words): header [64]: [0] magic [1] capacity the layout was made for
 //   [8 + 8 s ..] slot s: fill n (0xFFFFFFFF: none), P, A, ns;   [32 .. 45) zero between launches: scratch of the
-//   rank kernel's stage counts;   then slot 0, slot 1, each: tree [8192],
+//   rank kernel's stage counts;   then slot 0, slot 1, each: tree [32768],
 //   aux_1, aux_2, aux_3, buf (every array a multiple of 8 words long).
 // ---------------------------------------------------------------------------------------------
 constexpr int kIndexHeaderWords = 64;
@@ -520,9 +521,7 @@ struct IndexShape {
 __host__ __device__ inline IndexShape index_shape(int64_t n) {
   IndexShape s;
   s.A = 0;
-  while ((n >> (3 * (s.A + 1))) + 1 > (1 << kRankMaxTableLog2) - 1) ++s.A;
-  // a third aux level costs every candidate a fourth load from L2: a deeper tree is cheaper while it still fits
-  if (s.A == kIndexMaxLevels && (n >> (3 * kIndexMaxLevels)) + 1 <= (1 << kIndexMaxTreeLog2) - 1) --s.A;
+  while ((n >> (3 * (s.A + 1))) + 1 > (1 << kIndexMaxTreeLog2) - 1) ++s.A;
   s.ns = (int)(n >> (3 * (s.A + 1))) + 1;
   s.P = 1;
   while ((1 << s.P) - 1 < s.ns) ++s.P;

@@ -338,8 +338,8 @@ def _index_for(calib_dev, n, cap=None):
 
 @pytest.mark.parametrize("Nc,n", [(1 << 17, 8192), (100003, 8255), (1 << 16, 65536), (70001, 65543), (1 << 18, 327680),
                                    (16384, 524223), (20000, 100), (100, 70000), (0, 9000), (16384, 65527), (16384, 65528),
-                                   (1 << 16, 524224), (1 << 15, 4193791), (1 << 15, 4193792),
-                                   (1 << 15, 16776703), (1 << 15, 16776704)])
+                                   (1 << 16, 524224), (1 << 15, 262143), (1 << 15, 262144), (1 << 15, 2097151),
+                                   (1 << 15, 2097152), (1 << 15, 4193792), (1 << 15, 16776703), (1 << 15, 16777214)])
 def test_indexed_rank_equals_definition_and_plain_call(Nc, n):
     """The indexed rank gives the numerators and p-value bits of the definition, on smooth data, on heavily tied data
     and with special values at both ends of the buffer, with and without fused thresholds."""
