@@ -1387,23 +1387,30 @@ takeover_ids_kernel(const uint8_t* __restrict__ base, int64_t len, int head, int
 constexpr int kCondStage = 512;   // calibration entries a warp can stage in shared memory (2 KB)
 
 // Lower bound of four scores in their own segments [lo, lo + len) of `data` (shared memory), advanced together so
-// that the dependent loads overlap.
+// that the dependent loads overlap.  The halving form: while more than one entry is left, the first half of them
+// is dropped if its last entry is below the score; one comparison settles the last entry.  A step costs a load,
+// a comparison and a select, and leaves no length to keep besides the one count.
 __device__ __forceinline__ void lower_bound_four(const float* data, const float (&s)[4], int (&lo)[4], int (&len)[4]) {
-  const float qnan = __uint_as_float(0x7FC00000u);
-  while (max(max(len[0], len[1]), max(len[2], len[3])) > 0) {
-    float v[4];
+  int left[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = len[e] > 0 ? data[lo[e] + (len[e] >> 1)] : qnan;
+  for (int e = 0; e < 4; ++e) left[e] = len[e] > 0 ? len[e] : 0;
+  while (max(max(left[0], left[1]), max(left[2], left[3])) > 1) {
+    float v[4];
+    int half[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      if (len[e] > 0) {
-        const int half = len[e] >> 1;
-        const bool less = v[e] < s[e];
-        lo[e] = less ? lo[e] + half + 1 : lo[e];
-        len[e] = less ? len[e] - half - 1 : half;
-      }
+      half[e] = left[e] >> 1;   // 0 once at most one entry is left: nothing is read then
+      v[e] = half[e] > 0 ? data[lo[e] + half[e] - 1] : __uint_as_float(0x7FC00000u);
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      lo[e] += v[e] < s[e] ? half[e] : 0;   // NaN compares false
+      left[e] -= half[e];
     }
   }
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if (left[e] == 1 && data[lo[e]] < s[e]) lo[e] += 1;
 }
 
 // The same in global memory, for segments [lo, end) with len = end - lo entries (len <= 0: nothing to search).
