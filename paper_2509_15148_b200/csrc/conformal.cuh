@@ -997,25 +997,25 @@ merge_kernel(const float* __restrict__ old_buf, int n, const float* __restrict__
     // ---- place the own keys: e0 + #{tile entries <= x} + c_below + i ----
     for (int i = threadIdx.x; i < m; i += kMergeThreads) {
       const uint32_t x = own_sorted[i];
-      int p = 0, cnt = len;
-      while (cnt > 0) {
-        const int half = cnt >> 1;
-        const bool le = tkeys[p + half] <= x;
-        p = le ? p + half + 1 : p;
-        cnt = le ? cnt - half - 1 : half;
+      int p = 0, left = len;   // halving search: the first half goes if its last entry is not above x
+      while (left > 1) {
+        const int half = left >> 1;
+        p += (tkeys[p + half - 1] <= x) ? half : 0;
+        left -= half;
       }
+      if (left == 1 && tkeys[p] <= x) ++p;
       emit(e0 + p + c_below + i, x);
     }
     // ---- place the tile's old entries: e + c_below + #{own keys < old[e]} ----
     for (int i = threadIdx.x; i < len; i += kMergeThreads) {
       const uint32_t key = tkeys[i];
-      int p = 0, cnt = m;
-      while (cnt > 0) {
-        const int half = cnt >> 1;
-        const bool less = own_sorted[p + half] < key;
-        p = less ? p + half + 1 : p;
-        cnt = less ? cnt - half - 1 : half;
+      int p = 0, left = m;
+      while (left > 1) {
+        const int half = left >> 1;
+        p += (own_sorted[p + half - 1] < key) ? half : 0;
+        left -= half;
       }
+      if (left == 1 && own_sorted[p] < key) ++p;
       emit(e0 + i + c_below + p, key);
     }
     __syncthreads();   // shared memory is reused by the next tile
