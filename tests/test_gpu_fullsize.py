@@ -216,3 +216,31 @@ def test_conformal_stress_every_step_eager_with_index():
         n = n_next
     assert n == cap and np.all(np.diff(calib) >= 0)
     assert binding.last_device_status() == 0
+
+
+def test_takeover_ids_at_the_largest_range_size():
+    """Budget report on 2^24 + 3 stage bytes, where the kernel works in ranges of 32 KB over several turns per block:
+    mostly 10 % of the samples in stage 3, with a stretch in which all are (more positions than a range can stage: the
+    direct path), a stretch in which none is, other byte values, and a stage array that does not start on a 16-byte
+    boundary.  Expected positions by the definition, vectorised (numpy), which the oracle's loop is checked against on
+    a slice."""
+    Nc = (1 << 24) + 3
+    rng = np.random.default_rng(99)
+    stage_h = np.where(rng.random(Nc) < 0.1, 3, 2).astype(np.uint8)
+    stage_h[3_000_000:3_200_000] = 3
+    stage_h[9_000_000:9_300_000] = 2
+    stage_h[12_000_001:12_100_000] = rng.integers(0, 256, 99_999).astype(np.uint8)
+    want = np.flatnonzero(stage_h == 3).astype(np.int32)
+    assert np.array_equal(orc.takeover_ids(stage_h[2_990_000:3_010_000]) + 2_990_000, want[(want >= 2_990_000) & (want < 3_010_000)])
+    ws = workspace(binding.takeover_ids_workspace_bytes(Nc))
+    for shift in (0, 5):
+        st = poison((Nc + 16,), torch.uint8)
+        st[shift:shift + Nc] = dev(stage_h)
+        ids, count = poison((want.size + 3,), torch.int32), poison((1,), torch.int32)
+        binding.takeover_ids(st[shift:shift + Nc], ids[:want.size], count, ws)
+        torch.cuda.synchronize()
+        assert host_u32(count)[0] == want.size
+        got = ids.cpu().numpy()
+        assert np.array_equal(got[:want.size], want)
+        assert np.all(got.view(np.uint32)[want.size:] == 0xFFFFFFFF)
+    assert binding.last_device_status() == 0
