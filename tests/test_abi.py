@@ -68,6 +68,11 @@ def test_argument_errors_need_no_device():
     assert lib.atts_takeover_ids_workspace_bytes(-1, ctypes.byref(sz)) == 2
     assert lib.atts_takeover_ids(None, 8, None, 8, None, None, 0, None) == 1
     assert lib.atts_takeover_ids(None, 8, None, -1, None, None, 0, None) == 2
+    assert lib.atts_conformal_rank_conditional(None, None, 4, None, -1, None, 2, None, None, None, None) == 2   # array length
+    assert lib.atts_conformal_rank_conditional(None, None, 4, None, 1 << 31, None, 2, None, None, None, None) == 2
+    assert lib.atts_conformal_rank_conditional(None, None, 4, None, 10, None, 2, None, None, None, None) == 1
+    assert lib.atts_debug_set_wait(100, 2) == 6 and lib.atts_debug_set_wait(0, 0) == 0
+    assert lib.atts_debug_score_form(8, 100, 1000, None) == 1
     assert lib.atts_calib_index_build(None, 10, None, 0, None) == 1
     assert lib.atts_calib_index_build(None, 1 << 24, None, 0, None) == 2
     assert lib.atts_calib_update_indexed(None, 10, 20, None, 5, None, None, 0, None, 0, None) == 1
